@@ -1,0 +1,70 @@
+// Internal declarations shared by the host runtime and the kernel launchers.
+#pragma once
+
+#include <cstddef>
+#include <cstdint>
+#include <vector>
+
+#include "seqsched.h"
+
+namespace ss {
+
+// ---- scheduler (ss_sched.cpp) ------------------------------------------------------------
+int validate_sched_cfg(const ss_sched_cfg* c);
+int32_t length_bin(int32_t x, const ss_sched_cfg& c);
+int32_t batch_allowance(int32_t L, const ss_sched_cfg& c);
+int plan_first_pass(const ss_sched_cfg& c, const int32_t* prompt_len, const int32_t* pred_len,
+                    const int32_t* perm, int32_t n, std::vector<int32_t>& order,
+                    std::vector<ss_batch_desc>& out);
+
+// ---- constants ---------------------------------------------------------------------------
+constexpr int kPageTokens = 32;        // tokens per key/value page
+constexpr int kTileM = 128;            // weight rows per GEMM tile (tcgen05 M)
+constexpr int kTileK = 64;             // bf16 elements per 128-byte swizzled row
+constexpr int kAttnChunk = 256;        // tokens per decode-attention work item
+constexpr int kMaxBatch = 256;
+
+// Device status codes (which bounded wait expired / which check failed).
+enum : uint32_t {
+  kStatusOk = 0,
+  kStatusProducerTimeout = 1,
+  kStatusMmaTimeout = 2,
+  kStatusEpilogueTimeout = 3,
+  kStatusBadPage = 4,
+};
+
+// ---- GEMM:  D[n_out, tok] = W[n_out, K] . X[tok, K]^T  -------------------------------------
+// The tile-iteration space (n_tiles x kb) is cut into `gridx` equal contiguous ranges, one per
+// CTA (split along K where a range ends inside a tile).  In kGemmPartial mode every (CTA,
+// tile) segment is written as an fp32 partial; the consumer kernel adds the segments of a tile
+// in CTA order, so the result does not depend on timing.
+enum GemmMode : int { kGemmPartial = 0, kGemmDirectBf16 = 1, kGemmDirectF32Add = 2 };
+
+struct GemmPlan {
+  int n_out, K, n_tiles, kb;
+  int NT;              // token tile (tcgen05 N), multiple of 16, <= 256
+  int gridx, gridy;    // CTAs along the iteration space / token tiles
+  int max_seg;         // partial slots per CTA
+  int stages;
+  int smem_bytes;
+  int tmem_cols;
+};
+
+struct GemmArgs {
+  GemmPlan p;
+  int mode;
+  int n_tok;           // valid tokens
+  float* partial;      // [gridx*max_seg][NT][128]
+  void* out_bf16;      // [tok][ld_out]
+  float* out_f32;
+  int ld_out;
+  uint32_t* status;
+};
+
+// Partial-slot bookkeeping shared by the GEMM and its consumers.
+struct SplitInfo {
+  int gridx, kb, max_seg, NT;
+  long long total;     // n_tiles * kb
+};
+
+}  // namespace ss
