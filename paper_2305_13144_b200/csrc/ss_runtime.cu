@@ -1,0 +1,951 @@
+// Host runtime behind the C ABI: context, arena carve-up, weight repacking, key/value page
+// allocator, kernel sequencing (prompt pass, decode step, CUDA-graph replay) and the group loop
+// of Sec. 4.1 (micro-batches, caps, failure collection and recomputation).
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <map>
+#include <string>
+#include <vector>
+
+#include "ss_kernels.cuh"
+
+using namespace ss;
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+constexpr size_t kAlign = 1024;
+inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a; }
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+inline int round_up(int a, int b) { return ceil_div(a, b) * b; }
+
+struct LayerWeights {
+  bf16 *attn_norm, *wqkv, *wo, *ffn_norm, *wgu, *wdown;
+  CUtensorMap m_qkv, m_o, m_gu, m_down;
+};
+
+GemmPlan plan_gemm(int n_out, int K, int NT, int tok_tiles, int mode, int n_sm) {
+  GemmPlan p{};
+  p.n_out = n_out;
+  p.K = K;
+  p.n_tiles = ceil_div(n_out, kTileM);
+  p.kb = ceil_div(K, kTileK);
+  p.NT = NT;
+  const long long total = (long long)p.n_tiles * p.kb;
+  if (mode == kGemmPartial) {
+    p.gridx = (int)std::min<long long>(n_sm, total);
+    p.gridy = 1;
+  } else {
+    p.gridx = p.n_tiles;
+    p.gridy = tok_tiles;
+  }
+  const int ipc = (int)((total + p.gridx - 1) / p.gridx);
+  p.max_seg = (ipc + p.kb - 2) / p.kb + 1;
+  const int stage_bytes = kTileM * kTileK * 2 + NT * kTileK * 2;
+  const int budget = 227 * 1024 - 2048;                       // header + alignment slack
+  p.stages = std::max(2, std::min(kGemmMaxStages, budget / stage_bytes));
+  p.smem_bytes = 2048 + p.stages * stage_bytes;
+  int cols = 32;
+  while (cols < 2 * NT) cols <<= 1;
+  p.tmem_cols = cols;
+  return p;
+}
+
+SplitInfo split_of(const GemmPlan& p) {
+  SplitInfo s;
+  s.gridx = p.gridx;
+  s.kb = p.kb;
+  s.max_seg = p.max_seg;
+  s.NT = p.NT;
+  s.total = (long long)p.n_tiles * p.kb;
+  return s;
+}
+
+}  // namespace
+
+struct ss_ctx {
+  ss_model_cfg m;
+  ss_runtime_cfg rt;
+  cudaStream_t stream;
+  int n_sm = 148;
+  bool use_pdl = true;
+  int last_cuda = 0;
+  int64_t launches = 0;
+  bool capturing = false;
+  int64_t capture_count = 0;
+  EncodeTiledFn encode = nullptr;
+
+  // ---- arena
+  uint8_t* arena = nullptr;
+  size_t arena_bytes = 0;
+  // weights
+  bf16 *embed = nullptr, *lm_head = nullptr, *final_norm = nullptr;
+  std::vector<LayerWeights> layers;
+  CUtensorMap m_lm;
+  std::vector<uint8_t> loaded;     // per tensor slot
+  int n_loaded = 0, n_expected = 0;
+  // misc device
+  float* inv_freq = nullptr;
+  uint32_t* status = nullptr;
+  RowState st{};
+  KvLayout kv{};
+  int32_t *d_tokens = nullptr, *d_tok_row = nullptr, *d_tok_pos = nullptr, *d_cu = nullptr, *d_last = nullptr;
+  // prompt-pass activations (R rows)
+  int R = 0;
+  float* h = nullptr;
+  bf16 *x = nullptr, *qkv = nullptr, *attn_o = nullptr, *gu = nullptr, *act = nullptr;
+  // decode activations (kMaxBatch rows)
+  float* h_dec = nullptr;
+  bf16 *x_dec = nullptr, *q_dec = nullptr, *o_dec = nullptr, *act_dec = nullptr;
+  float* partial = nullptr;
+  size_t partial_bytes = 0;
+  float *part_ml = nullptr, *part_acc = nullptr;
+  int max_chunks = 0;
+  // tensor maps for activation operands, keyed by (buffer id, box rows)
+  std::map<std::pair<int, int>, CUtensorMap> xmaps;
+
+  // ---- page allocator
+  std::vector<int32_t> free_pages;
+  std::vector<int32_t> batch_pages;
+
+  // ---- batch state (host mirror)
+  int B = 0;
+  int cap = 0;
+  bool in_batch = false;
+  std::vector<int32_t> prompt_len;
+  int32_t* pinned = nullptr;     // [0] n_active, [1] status
+  std::map<int, cudaGraphExec_t> graphs;   // decode step per batch size
+  int64_t graph_nodes = 0;
+};
+
+namespace {
+
+int cuda_fail(ss_ctx* c, cudaError_t e) {
+  c->last_cuda = (int)e;
+  return SS_ERR_CUDA;
+}
+#define SS_CUDA(c, expr)                                \
+  do {                                                  \
+    cudaError_t _e = (expr);                            \
+    if (_e != cudaSuccess) return cuda_fail((c), _e);   \
+  } while (0)
+
+template <class... KArgs, class... Args>
+cudaError_t launch(ss_ctx* c, void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, Args... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = c->stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = c->use_pdl ? 1 : 0;
+  if (c->capturing) c->capture_count++; else c->launches++;
+  return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
+}
+
+int make_map(ss_ctx* c, CUtensorMap* out, const void* base, int64_t rows, int64_t cols, int box_rows) {
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {(cuuint32_t)kTileK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = c->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    c->last_cuda = (int)r;
+    return SS_ERR_CUDA;
+  }
+  return SS_OK;
+}
+
+// activation operand map (cached): id 0 = x, 1 = attn_o, 2 = act (prompt pass); 3 = x_dec, 4 = o_dec, 5 = act_dec
+int xmap(ss_ctx* c, int id, int box_rows, const CUtensorMap** out) {
+  auto key = std::make_pair(id, box_rows);
+  auto it = c->xmaps.find(key);
+  if (it == c->xmaps.end()) {
+    const int d = c->m.d_model, F = c->m.d_ffn;
+    const void* base = nullptr;
+    int64_t rows = 0, cols = 0;
+    switch (id) {
+      case 0: base = c->x; rows = c->R; cols = d; break;
+      case 1: base = c->attn_o; rows = c->R; cols = d; break;
+      case 2: base = c->act; rows = c->R; cols = F; break;
+      case 3: base = c->x_dec; rows = kMaxBatch; cols = d; break;
+      case 4: base = c->o_dec; rows = kMaxBatch; cols = d; break;
+      default: base = c->act_dec; rows = kMaxBatch; cols = F; break;
+    }
+    CUtensorMap m;
+    int rc = make_map(c, &m, base, rows, cols, box_rows);
+    if (rc != SS_OK) return rc;
+    it = c->xmaps.emplace(key, m).first;
+  }
+  *out = &it->second;
+  return SS_OK;
+}
+
+int run_gemm(ss_ctx* c, const CUtensorMap& mw, const CUtensorMap& mx, const GemmPlan& p, int mode, int n_tok,
+             void* out_bf16, float* out_f32, int ld_out) {
+  GemmArgs a{};
+  a.p = p;
+  a.mode = mode;
+  a.n_tok = n_tok;
+  a.partial = c->partial;
+  a.out_bf16 = out_bf16;
+  a.out_f32 = out_f32;
+  a.ld_out = ld_out;
+  a.status = c->status;
+  if (mode == kGemmPartial) {
+    const size_t need = (size_t)p.gridx * p.max_seg * p.NT * 128 * sizeof(float);
+    if (need > c->partial_bytes) return SS_ERR_CAPACITY;
+  }
+  SS_CUDA(c, launch(c, gemm_wx_kernel, dim3(p.gridy, p.gridx), dim3(kGemmThreads), (size_t)p.smem_bytes, mw, mx, a));
+  return SS_OK;
+}
+
+struct ArenaPlan {
+  size_t total = 0;
+  size_t take(size_t bytes) {
+    size_t off = total;
+    total = align_up(total + bytes);
+    return off;
+  }
+};
+
+struct Offsets {
+  size_t embed, lm_head, final_norm;
+  std::vector<size_t> attn_norm, wqkv, wo, ffn_norm, wgu, wdown;
+  size_t inv_freq, status, rows, block_table, out_tokens, tok, h, x, qkv, attn_o, gu, act;
+  size_t h_dec, x_dec, q_dec, o_dec, act_dec, partial, part_ml, part_acc, kv;
+  size_t partial_bytes;
+  int R, max_pages, n_pages, max_chunks;
+  size_t total;
+};
+
+int validate_model(const ss_model_cfg* m, const ss_runtime_cfg* rt) {
+  if (!m || !rt) return SS_ERR_ARG;
+  if (m->n_layers < 0 || m->d_model <= 0 || m->n_heads <= 0 || m->d_ffn <= 0 || m->vocab <= 0) return SS_ERR_ARG;
+  if (m->eos_id < 0 || m->eos_id >= m->vocab) return SS_ERR_ARG;
+  if (m->n_heads * m->head_dim != m->d_model) return SS_ERR_ARG;
+  if (m->head_dim != 64 && m->head_dim != 128) return SS_ERR_UNSUPPORTED;
+  if (m->d_model % 64 || m->d_model > 8192 || m->d_ffn % 8) return SS_ERR_UNSUPPORTED;
+  if (rt->max_batch < 1 || rt->max_batch > kMaxBatch) return SS_ERR_ARG;
+  if (rt->max_ctx < 2 || rt->max_prefill_tokens < 1 || rt->max_new_tokens < 1 || rt->kv_pool_tokens < 1) return SS_ERR_ARG;
+  return SS_OK;
+}
+
+void layout(const ss_model_cfg& m, const ss_runtime_cfg& rt, int n_sm, Offsets& o) {
+  ArenaPlan a;
+  const size_t d = m.d_model, F = m.d_ffn, V = m.vocab;
+  o.embed = a.take(V * d * 2);
+  o.attn_norm.resize(m.n_layers); o.wqkv.resize(m.n_layers); o.wo.resize(m.n_layers);
+  o.ffn_norm.resize(m.n_layers); o.wgu.resize(m.n_layers); o.wdown.resize(m.n_layers);
+  for (int l = 0; l < m.n_layers; ++l) {
+    o.attn_norm[l] = a.take(d * 2);
+    o.wqkv[l] = a.take(3 * d * d * 2);
+    o.wo[l] = a.take(d * d * 2);
+    o.ffn_norm[l] = a.take(d * 2);
+    o.wgu[l] = a.take(2 * F * d * 2);
+    o.wdown[l] = a.take(d * F * 2);
+  }
+  o.final_norm = a.take(d * 2);
+  o.lm_head = a.take(V * d * 2);
+  o.inv_freq = a.take(m.head_dim / 2 * sizeof(float));
+  o.status = a.take(64);
+  o.rows = a.take((size_t)kMaxBatch * 4 * 8 + 64);           // 7 row arrays + scalars
+  o.max_pages = ceil_div(rt.max_ctx, kPageTokens);
+  o.block_table = a.take((size_t)kMaxBatch * o.max_pages * 4);
+  o.out_tokens = a.take((size_t)kMaxBatch * rt.max_new_tokens * 4);
+  o.R = round_up(std::max(rt.max_prefill_tokens, kMaxBatch), 256);
+  o.tok = a.take(((size_t)o.R * 3 + 2 * kMaxBatch + 8) * 4);
+  o.h = a.take((size_t)o.R * d * 4);
+  o.x = a.take((size_t)o.R * d * 2);
+  o.qkv = a.take((size_t)o.R * 3 * d * 2);
+  o.attn_o = a.take((size_t)o.R * d * 2);
+  o.gu = a.take((size_t)o.R * 2 * F * 2);
+  o.act = a.take((size_t)o.R * F * 2);
+  o.h_dec = a.take((size_t)kMaxBatch * d * 4);
+  o.x_dec = a.take((size_t)kMaxBatch * d * 2);
+  o.q_dec = a.take((size_t)kMaxBatch * d * 2);
+  o.o_dec = a.take((size_t)kMaxBatch * d * 2);
+  o.act_dec = a.take((size_t)kMaxBatch * F * 2);
+  // partial work space: the largest decode GEMM at the widest token tile
+  const int NTmax = round_up(rt.max_batch, 16);
+  size_t pb = 0;
+  const int shapes[5][2] = {{(int)(3 * d), (int)d}, {(int)d, (int)d}, {(int)(2 * F), (int)d}, {(int)d, (int)F}, {(int)V, (int)d}};
+  for (auto& s : shapes) {
+    GemmPlan p = plan_gemm(s[0], s[1], NTmax, 1, kGemmPartial, n_sm);
+    pb = std::max(pb, (size_t)p.gridx * p.max_seg * p.NT * 128 * sizeof(float));
+  }
+  o.partial_bytes = pb;
+  o.partial = a.take(pb);
+  o.max_chunks = ceil_div(rt.max_ctx, kAttnChunk);
+  o.part_ml = a.take((size_t)kMaxBatch * m.n_heads * o.max_chunks * 2 * 4);
+  o.part_acc = a.take((size_t)kMaxBatch * m.n_heads * o.max_chunks * m.head_dim * 4);
+  o.n_pages = (int)((rt.kv_pool_tokens + kPageTokens - 1) / kPageTokens) + rt.max_batch;
+  const size_t page_bytes = (size_t)2 * m.n_heads * kPageTokens * m.head_dim * 2;
+  o.kv = a.take((size_t)std::max(1, m.n_layers) * o.n_pages * page_bytes);
+  o.total = a.total;
+}
+
+int query_sms() {
+  int dev = 0, n = 148;
+  if (cudaGetDevice(&dev) == cudaSuccess) {
+    int v = 0;
+    if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && v > 0) n = v;
+  }
+  return n;
+}
+
+int weight_slot(const ss_ctx* c, const std::string& name, bf16** dst, int64_t* rows, int64_t* cols, int* slot) {
+  const int64_t d = c->m.d_model, F = c->m.d_ffn, V = c->m.vocab;
+  auto set = [&](bf16* p, int64_t r, int64_t cc, int s) { *dst = p; *rows = r; *cols = cc; *slot = s; return SS_OK; };
+  if (name == "embed") return set(c->embed, V, d, 0);
+  if (name == "lm_head") return set(c->lm_head, V, d, 1);
+  if (name == "final_norm") return set(c->final_norm, 1, d, 2);
+  if (name.size() > 2 && name[0] == 'l') {
+    size_t dot = name.find('.');
+    if (dot == std::string::npos) return SS_ERR_ARG;
+    int l = atoi(name.substr(1, dot - 1).c_str());
+    if (l < 0 || l >= c->m.n_layers) return SS_ERR_ARG;
+    const std::string k = name.substr(dot + 1);
+    const LayerWeights& w = c->layers[l];
+    const int base = 3 + l * 9;
+    if (k == "attn_norm") return set(w.attn_norm, 1, d, base + 0);
+    if (k == "wq") return set(w.wqkv, d, d, base + 1);
+    if (k == "wk") return set(w.wqkv + d * d, d, d, base + 2);
+    if (k == "wv") return set(w.wqkv + 2 * d * d, d, d, base + 3);
+    if (k == "wo") return set(w.wo, d, d, base + 4);
+    if (k == "ffn_norm") return set(w.ffn_norm, 1, d, base + 5);
+    if (k == "w_gate") return set(w.wgu, F, d, base + 6);
+    if (k == "w_up") return set(w.wgu + F * d, F, d, base + 7);
+    if (k == "w_down") return set(w.wdown, d, F, base + 8);
+  }
+  return SS_ERR_ARG;
+}
+
+double weight_bytes_per_step(const ss_model_cfg& m) {
+  const double d = m.d_model, F = m.d_ffn, V = m.vocab;
+  return m.n_layers * (4 * d * d + 3 * d * F + 2 * d) * 2.0 + V * d * 2.0 + d * 2.0;
+}
+double kv_bytes_per_token(const ss_model_cfg& m) { return 2.0 * m.d_model * 2.0 * m.n_layers; }
+
+// ------------------------------------------------------------------------------------ decode step
+int enqueue_decode_step(ss_ctx* c, const ss_step_opts* opts, int32_t* next_tokens) {
+  const ss_model_cfg& m = c->m;
+  const int B = c->B, d = m.d_model, F = m.d_ffn, H = m.n_heads, Dh = m.head_dim, V = m.vocab;
+  const int NT = round_up(B, 16);
+  const CUtensorMap *mx, *mo, *ma;
+  int rc;
+  if ((rc = xmap(c, 3, NT, &mx)) || (rc = xmap(c, 4, NT, &mo)) || (rc = xmap(c, 5, NT, &ma))) return rc;
+  const GemmPlan p_qkv = plan_gemm(3 * d, d, NT, 1, kGemmPartial, c->n_sm);
+  const GemmPlan p_o = plan_gemm(d, d, NT, 1, kGemmPartial, c->n_sm);
+  const GemmPlan p_gu = plan_gemm(2 * F, d, NT, 1, kGemmPartial, c->n_sm);
+  const GemmPlan p_dn = plan_gemm(d, F, NT, 1, kGemmPartial, c->n_sm);
+  const GemmPlan p_lm = plan_gemm(V, d, NT, 1, kGemmPartial, c->n_sm);
+  const bf16* first_norm = m.n_layers ? c->layers[0].attn_norm : c->final_norm;
+  SS_CUDA(c, launch(c, embed_rmsnorm_kernel, dim3(B), dim3(256), 0, (const int32_t*)c->st.cur_tok,
+                    (const int32_t*)c->st.active, (const bf16*)c->embed, first_norm, c->h_dec, c->x_dec, d, m.rms_eps, V));
+  AttnArgs aa{};
+  aa.st = c->st; aa.kv = c->kv; aa.q = c->q_dec; aa.part_ml = c->part_ml; aa.part_acc = c->part_acc;
+  aa.out = c->o_dec; aa.B = B; aa.d = d; aa.max_chunks = c->max_chunks; aa.status = c->status;
+  const int attn_grid = c->n_sm * 4;
+  for (int l = 0; l < m.n_layers; ++l) {
+    const LayerWeights& w = c->layers[l];
+    if ((rc = run_gemm(c, w.m_qkv, *mx, p_qkv, kGemmPartial, B, nullptr, nullptr, 0))) return rc;
+    SS_CUDA(c, launch(c, rope_append_decode_kernel, dim3(H, B), dim3(Dh / 2), 0, (const float*)c->partial,
+                      split_of(p_qkv), c->st, c->kv, l, (const float*)c->inv_freq, c->q_dec, d, c->status));
+    aa.layer = l;
+    if (Dh == 128) {
+      SS_CUDA(c, launch(c, attn_decode_kernel<128>, dim3(attn_grid), dim3(128), 0, aa));
+      SS_CUDA(c, launch(c, attn_combine_kernel<128>, dim3(H, B), dim3(128), 0, aa));
+    } else {
+      SS_CUDA(c, launch(c, attn_decode_kernel<64>, dim3(attn_grid), dim3(128), 0, aa));
+      SS_CUDA(c, launch(c, attn_combine_kernel<64>, dim3(H, B), dim3(64), 0, aa));
+    }
+    if ((rc = run_gemm(c, w.m_o, *mo, p_o, kGemmPartial, B, nullptr, nullptr, 0))) return rc;
+    SS_CUDA(c, launch(c, residual_rmsnorm_partial_kernel, dim3(B), dim3(256), 0, (const float*)c->partial,
+                      split_of(p_o), (const int32_t*)c->st.active, c->h_dec, (const bf16*)w.ffn_norm, c->x_dec,
+                      (float*)nullptr, d, m.rms_eps));
+    if ((rc = run_gemm(c, w.m_gu, *mx, p_gu, kGemmPartial, B, nullptr, nullptr, 0))) return rc;
+    SS_CUDA(c, launch(c, swiglu_partial_kernel, dim3(ceil_div(F, 256), B), dim3(256), 0, (const float*)c->partial,
+                      split_of(p_gu), c->act_dec, F));
+    if ((rc = run_gemm(c, w.m_down, *ma, p_dn, kGemmPartial, B, nullptr, nullptr, 0))) return rc;
+    const bool last = l + 1 == m.n_layers;
+    const bf16* next_norm = last ? c->final_norm : c->layers[l + 1].attn_norm;
+    SS_CUDA(c, launch(c, residual_rmsnorm_partial_kernel, dim3(B), dim3(256), 0, (const float*)c->partial,
+                      split_of(p_dn), (const int32_t*)c->st.active, c->h_dec, next_norm, c->x_dec,
+                      (last && opts) ? opts->dump_hidden : (float*)nullptr, d, m.rms_eps));
+  }
+  if (m.n_layers == 0 && opts && opts->dump_hidden)
+    SS_CUDA(c, cudaMemcpyAsync(opts->dump_hidden, c->h_dec, (size_t)B * d * 4, cudaMemcpyDeviceToDevice, c->stream));
+  if ((rc = run_gemm(c, c->m_lm, *mx, p_lm, kGemmPartial, B, nullptr, nullptr, 0))) return rc;
+  SS_CUDA(c, launch(c, lmhead_argmax_kernel, dim3(B), dim3(1024), 0, (const float*)c->partial, split_of(p_lm), c->st,
+                    opts ? opts->dump_logits : (float*)nullptr, V, m.eos_id));
+  SS_CUDA(c, launch(c, bookkeeping_kernel, dim3(1), dim3(kMaxBatch), 0, c->st,
+                    opts ? opts->forced_tokens : (const int32_t*)nullptr, next_tokens, B, m.eos_id, 0));
+  return SS_OK;
+}
+
+// ------------------------------------------------------------------------------------ prompt pass (one chunk of whole sequences)
+int enqueue_prefill_chunk(ss_ctx* c, int s0, int s1, const int32_t* cu, int T) {
+  const ss_model_cfg& m = c->m;
+  const int d = m.d_model, F = m.d_ffn, H = m.n_heads, Dh = m.head_dim, V = m.vocab;
+  const int nseq = s1 - s0;
+  int max_len = 0;
+  for (int s = s0; s < s1; ++s) max_len = std::max(max_len, cu[s + 1] - cu[s]);
+  const int NT = std::min(256, round_up(T, 16));
+  const int tok_tiles = ceil_div(T, NT);
+  const CUtensorMap *mx, *mo, *ma;
+  int rc;
+  if ((rc = xmap(c, 0, NT, &mx)) || (rc = xmap(c, 1, NT, &mo)) || (rc = xmap(c, 2, NT, &ma))) return rc;
+  const GemmPlan p_qkv = plan_gemm(3 * d, d, NT, tok_tiles, kGemmDirectBf16, c->n_sm);
+  const GemmPlan p_o = plan_gemm(d, d, NT, tok_tiles, kGemmDirectF32Add, c->n_sm);
+  const GemmPlan p_gu = plan_gemm(2 * F, d, NT, tok_tiles, kGemmDirectBf16, c->n_sm);
+  const GemmPlan p_dn = plan_gemm(d, F, NT, tok_tiles, kGemmDirectF32Add, c->n_sm);
+  const bf16* first_norm = m.n_layers ? c->layers[0].attn_norm : c->final_norm;
+  SS_CUDA(c, launch(c, embed_rmsnorm_kernel, dim3(T), dim3(256), 0, (const int32_t*)c->d_tokens, (const int32_t*)nullptr,
+                    (const bf16*)c->embed, first_norm, c->h, c->x, d, m.rms_eps, V));
+  for (int l = 0; l < m.n_layers; ++l) {
+    const LayerWeights& w = c->layers[l];
+    if ((rc = run_gemm(c, w.m_qkv, *mx, p_qkv, kGemmDirectBf16, T, c->qkv, nullptr, 3 * d))) return rc;
+    SS_CUDA(c, launch(c, rope_append_prefill_kernel, dim3(T, H), dim3(Dh / 2), 0, c->qkv, (const int32_t*)c->d_tok_row,
+                      (const int32_t*)c->d_tok_pos, c->st, c->kv, l, (const float*)c->inv_freq, d, c->status));
+    const dim3 ag(ceil_div(max_len, 32), H, nseq);
+    if (Dh == 128)
+      SS_CUDA(c, launch(c, attn_prefill_kernel<128>, ag, dim3(128), 0, (const bf16*)c->qkv, (const int32_t*)c->d_cu, c->attn_o, d));
+    else
+      SS_CUDA(c, launch(c, attn_prefill_kernel<64>, ag, dim3(128), 0, (const bf16*)c->qkv, (const int32_t*)c->d_cu, c->attn_o, d));
+    if ((rc = run_gemm(c, w.m_o, *mo, p_o, kGemmDirectF32Add, T, nullptr, c->h, d))) return rc;
+    SS_CUDA(c, launch(c, rmsnorm_kernel, dim3(T), dim3(256), 0, (const float*)c->h, (const bf16*)w.ffn_norm, c->x, d, m.rms_eps));
+    if ((rc = run_gemm(c, w.m_gu, *mx, p_gu, kGemmDirectBf16, T, c->gu, nullptr, 2 * F))) return rc;
+    SS_CUDA(c, launch(c, swiglu_kernel, dim3(T, ceil_div(F, 256)), dim3(256), 0, (const bf16*)c->gu, c->act, F));
+    if ((rc = run_gemm(c, w.m_down, *ma, p_dn, kGemmDirectF32Add, T, nullptr, c->h, d))) return rc;
+    if (l + 1 < m.n_layers)
+      SS_CUDA(c, launch(c, rmsnorm_kernel, dim3(T), dim3(256), 0, (const float*)c->h,
+                        (const bf16*)c->layers[l + 1].attn_norm, c->x, d, m.rms_eps));
+  }
+  return SS_OK;
+}
+
+}  // namespace
+
+// ======================================================================================= C ABI
+extern "C" {
+
+const char* ss_strerror(int code) {
+  switch (code) {
+    case SS_OK: return "ok";
+    case SS_ERR_ARG: return "bad argument";
+    case SS_ERR_CAPACITY: return "buffer or arena too small";
+    case SS_ERR_KV_BUDGET: return "batch does not fit the key/value pool";
+    case SS_ERR_STATE: return "call out of order";
+    case SS_ERR_CUDA: return "CUDA call failed";
+    case SS_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel expired";
+    case SS_ERR_UNSUPPORTED: return "shape not supported by the kernels";
+    default: return "unknown error";
+  }
+}
+
+int ss_arena_bytes(const ss_model_cfg* model, const ss_runtime_cfg* rt, size_t* out_bytes) {
+  int rc = validate_model(model, rt);
+  if (rc) return rc;
+  if (!out_bytes) return SS_ERR_ARG;
+  Offsets o;
+  layout(*model, *rt, 148, o);          // sized for the largest grid the kernels use
+  *out_bytes = o.total;
+  return SS_OK;
+}
+
+int ss_create(const ss_model_cfg* model, const ss_runtime_cfg* rt, void* dev_arena, size_t arena_bytes, void* stream,
+              ss_ctx** out) {
+  int rc = validate_model(model, rt);
+  if (rc) return rc;
+  if (!dev_arena || !out || ((uintptr_t)dev_arena % kAlign)) return SS_ERR_ARG;
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) return SS_ERR_CUDA;
+  Offsets o;
+  layout(*model, *rt, 148, o);
+  if (arena_bytes < o.total) return SS_ERR_CAPACITY;
+  ss_ctx* c = new ss_ctx();
+  c->m = *model;
+  c->rt = *rt;
+  c->stream = (cudaStream_t)stream;
+  c->n_sm = std::min(148, query_sms());
+  c->use_pdl = getenv("SS_NO_PDL") == nullptr;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qr;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qr) != cudaSuccess || !fn) {
+    delete c;
+    return SS_ERR_CUDA;
+  }
+  c->encode = (EncodeTiledFn)fn;
+  uint8_t* A = (uint8_t*)dev_arena;
+  c->arena = A;
+  c->arena_bytes = arena_bytes;
+  const int64_t d = model->d_model, F = model->d_ffn, V = model->vocab;
+  c->embed = (bf16*)(A + o.embed);
+  c->lm_head = (bf16*)(A + o.lm_head);
+  c->final_norm = (bf16*)(A + o.final_norm);
+  c->layers.resize(model->n_layers);
+  auto fail = [&](int code) { delete c; return code; };
+  for (int l = 0; l < model->n_layers; ++l) {
+    LayerWeights& w = c->layers[l];
+    w.attn_norm = (bf16*)(A + o.attn_norm[l]);
+    w.wqkv = (bf16*)(A + o.wqkv[l]);
+    w.wo = (bf16*)(A + o.wo[l]);
+    w.ffn_norm = (bf16*)(A + o.ffn_norm[l]);
+    w.wgu = (bf16*)(A + o.wgu[l]);
+    w.wdown = (bf16*)(A + o.wdown[l]);
+    if ((rc = make_map(c, &w.m_qkv, w.wqkv, 3 * d, d, kTileM))) return fail(rc);
+    if ((rc = make_map(c, &w.m_o, w.wo, d, d, kTileM))) return fail(rc);
+    if ((rc = make_map(c, &w.m_gu, w.wgu, 2 * F, d, kTileM))) return fail(rc);
+    if ((rc = make_map(c, &w.m_down, w.wdown, d, F, kTileM))) return fail(rc);
+  }
+  if ((rc = make_map(c, &c->m_lm, c->lm_head, V, d, kTileM))) return fail(rc);
+  c->n_expected = 3 + 9 * model->n_layers;
+  c->loaded.assign(c->n_expected, 0);
+  c->inv_freq = (float*)(A + o.inv_freq);
+  c->status = (uint32_t*)(A + o.status);
+  int32_t* rows = (int32_t*)(A + o.rows);
+  c->st.ctx_len = rows + 0 * kMaxBatch;
+  c->st.cur_tok = rows + 1 * kMaxBatch;
+  c->st.gen = rows + 2 * kMaxBatch;
+  c->st.active = rows + 3 * kMaxBatch;
+  c->st.finished = rows + 4 * kMaxBatch;
+  c->st.eos_at = rows + 5 * kMaxBatch;
+  c->st.choice = rows + 6 * kMaxBatch;
+  c->st.scalars = rows + 7 * kMaxBatch;
+  c->st.block_table = (int32_t*)(A + o.block_table);
+  c->st.out_tokens = (int32_t*)(A + o.out_tokens);
+  c->st.max_pages = o.max_pages;
+  c->st.max_new = rt->max_new_tokens;
+  c->R = o.R;
+  int32_t* tk = (int32_t*)(A + o.tok);
+  c->d_tokens = tk;
+  c->d_tok_row = tk + o.R;
+  c->d_tok_pos = tk + 2 * (size_t)o.R;
+  c->d_cu = tk + 3 * (size_t)o.R;
+  c->d_last = c->d_cu + kMaxBatch + 4;
+  c->h = (float*)(A + o.h);
+  c->x = (bf16*)(A + o.x);
+  c->qkv = (bf16*)(A + o.qkv);
+  c->attn_o = (bf16*)(A + o.attn_o);
+  c->gu = (bf16*)(A + o.gu);
+  c->act = (bf16*)(A + o.act);
+  c->h_dec = (float*)(A + o.h_dec);
+  c->x_dec = (bf16*)(A + o.x_dec);
+  c->q_dec = (bf16*)(A + o.q_dec);
+  c->o_dec = (bf16*)(A + o.o_dec);
+  c->act_dec = (bf16*)(A + o.act_dec);
+  c->partial = (float*)(A + o.partial);
+  c->partial_bytes = o.partial_bytes;
+  c->part_ml = (float*)(A + o.part_ml);
+  c->part_acc = (float*)(A + o.part_acc);
+  c->max_chunks = o.max_chunks;
+  c->kv.pool = (bf16*)(A + o.kv);
+  c->kv.page_elems = (size_t)2 * model->n_heads * kPageTokens * model->head_dim;
+  c->kv.layer_stride = (size_t)o.n_pages * c->kv.page_elems;
+  c->kv.n_pages = o.n_pages;
+  c->kv.H = model->n_heads;
+  c->kv.Dh = model->head_dim;
+  c->free_pages.resize(o.n_pages);
+  for (int i = 0; i < o.n_pages; ++i) c->free_pages[i] = o.n_pages - 1 - i;
+
+  // rotary inverse frequencies, exact in double then rounded once
+  std::vector<float> inv(model->head_dim / 2);
+  for (int i = 0; i < model->head_dim / 2; ++i)
+    inv[i] = (float)std::pow((double)model->rope_theta, -2.0 * i / model->head_dim);
+  cudaError_t e = cudaMemcpyAsync(c->inv_freq, inv.data(), inv.size() * 4, cudaMemcpyHostToDevice, c->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(c->status, 0, 64, c->stream);
+  if (e == cudaSuccess) e = cudaMemsetAsync(rows, 0, (size_t)kMaxBatch * 4 * 8 + 64, c->stream);
+  // activation operands must be finite wherever a TMA box may reach beyond the valid rows
+  if (e == cudaSuccess) e = cudaMemsetAsync(A + o.h, 0, o.partial - o.h, c->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);
+  if (e == cudaSuccess) e = cudaHostAlloc((void**)&c->pinned, 64, cudaHostAllocDefault);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(gemm_wx_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e != cudaSuccess) {
+    c->last_cuda = (int)e;
+    delete c;
+    return SS_ERR_CUDA;
+  }
+  *out = c;
+  return SS_OK;
+}
+
+int ss_destroy(ss_ctx* c) {
+  if (!c) return SS_ERR_ARG;
+  cudaStreamSynchronize(c->stream);
+  for (auto& g : c->graphs) cudaGraphExecDestroy(g.second);
+  if (c->pinned) cudaFreeHost(c->pinned);
+  delete c;
+  return SS_OK;
+}
+
+int ss_load_weights(ss_ctx* c, const ss_tensor_desc* t, int32_t n) {
+  if (!c || (n > 0 && !t) || n < 0) return SS_ERR_ARG;
+  for (int i = 0; i < n; ++i) {
+    if (!t[i].name || !t[i].data) return SS_ERR_ARG;
+    bf16* dst;
+    int64_t rows, cols;
+    int slot;
+    int rc = weight_slot(c, t[i].name, &dst, &rows, &cols, &slot);
+    if (rc) return rc;
+    if (t[i].rows * t[i].cols != rows * cols || (rows > 1 && (t[i].rows != rows || t[i].cols != cols))) return SS_ERR_ARG;
+    SS_CUDA(c, cudaMemcpyAsync(dst, t[i].data, (size_t)rows * cols * 2,
+                               t[i].is_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, c->stream));
+    if (!c->loaded[slot]) { c->loaded[slot] = 1; c->n_loaded++; }
+  }
+  SS_CUDA(c, cudaStreamSynchronize(c->stream));
+  return SS_OK;
+}
+
+int ss_release_batch(ss_ctx* c) {
+  if (!c) return SS_ERR_ARG;
+  for (int32_t p : c->batch_pages) c->free_pages.push_back(p);
+  c->batch_pages.clear();
+  c->in_batch = false;
+  c->B = 0;
+  return SS_OK;
+}
+
+int ss_prefill(ss_ctx* c, const int32_t* tokens, const int32_t* cu, int32_t B, const int32_t* eos_at, int32_t cap,
+               const ss_step_opts* opts, int32_t* first_tokens) {
+  if (!c || !tokens || !cu || B < 1 || cap < 1) return SS_ERR_ARG;
+  if (c->n_loaded != c->n_expected || c->in_batch) return SS_ERR_STATE;
+  if (B > c->rt.max_batch || cap > c->rt.max_new_tokens) return SS_ERR_CAPACITY;
+  if (cu[0] != 0) return SS_ERR_ARG;
+  const ss_model_cfg& m = c->m;
+  // admission: pages for the worst case of every row
+  size_t need_pages = 0;
+  for (int r = 0; r < B; ++r) {
+    const int len = cu[r + 1] - cu[r];
+    if (len < 1) return SS_ERR_ARG;
+    if (len > c->rt.max_prefill_tokens || len + cap > c->rt.max_ctx) return SS_ERR_CAPACITY;
+    need_pages += ceil_div(len + cap, kPageTokens);
+    if (eos_at && eos_at[r] < 1) return SS_ERR_ARG;
+  }
+  if (need_pages > c->free_pages.size()) return SS_ERR_KV_BUDGET;
+  const int Ttot = cu[B];
+  for (int i = 0; i < Ttot; ++i)
+    if (tokens[i] < 0 || tokens[i] >= m.vocab) return SS_ERR_ARG;
+
+  // host-side batch state
+  std::vector<int32_t> bt((size_t)B * c->st.max_pages, -1);
+  c->batch_pages.clear();
+  c->prompt_len.assign(B, 0);
+  for (int r = 0; r < B; ++r) {
+    const int len = cu[r + 1] - cu[r];
+    c->prompt_len[r] = len;
+    const int np = ceil_div(len + cap, kPageTokens);
+    for (int p = 0; p < np; ++p) {
+      const int32_t pg = c->free_pages.back();
+      c->free_pages.pop_back();
+      c->batch_pages.push_back(pg);
+      bt[(size_t)r * c->st.max_pages + p] = pg;
+    }
+  }
+  c->in_batch = true;
+  c->B = B;
+  c->cap = cap;
+  std::vector<int32_t> rows((size_t)kMaxBatch * 8, 0);
+  for (int r = 0; r < B; ++r) {
+    rows[0 * kMaxBatch + r] = c->prompt_len[r];   // ctx_len after the prompt pass
+    rows[3 * kMaxBatch + r] = 1;                  // active
+    rows[5 * kMaxBatch + r] = eos_at ? eos_at[r] : 0;
+  }
+  rows[7 * kMaxBatch + 0] = cap;
+  rows[7 * kMaxBatch + 1] = B;
+  int rc = SS_OK;
+  auto bail = [&](int code) { ss_release_batch(c); return code; };
+#define SS_CUDA_B(expr)                                              \
+  do {                                                               \
+    cudaError_t _e = (expr);                                         \
+    if (_e != cudaSuccess) { c->last_cuda = (int)_e; return bail(SS_ERR_CUDA); } \
+  } while (0)
+  SS_CUDA_B(cudaMemcpyAsync(c->st.ctx_len, rows.data(), rows.size() * 4, cudaMemcpyHostToDevice, c->stream));
+  SS_CUDA_B(cudaMemcpyAsync(c->st.block_table, bt.data(), bt.size() * 4, cudaMemcpyHostToDevice, c->stream));
+
+  // chunks of whole sequences
+  std::vector<int32_t> tok_row, tok_pos, cu_loc, last;
+  int s0 = 0;
+  while (s0 < B) {
+    int s1 = s0, T = 0;
+    while (s1 < B && T + (cu[s1 + 1] - cu[s1]) <= c->rt.max_prefill_tokens) { T += cu[s1 + 1] - cu[s1]; ++s1; }
+    tok_row.resize(T); tok_pos.resize(T); cu_loc.assign(1, 0); last.clear();
+    int t = 0;
+    for (int s = s0; s < s1; ++s) {
+      const int len = cu[s + 1] - cu[s];
+      for (int p = 0; p < len; ++p, ++t) { tok_row[t] = s; tok_pos[t] = p; }
+      cu_loc.push_back(t);
+      last.push_back(t - 1);
+    }
+    SS_CUDA_B(cudaMemcpyAsync(c->d_tokens, tokens + cu[s0], (size_t)T * 4, cudaMemcpyHostToDevice, c->stream));
+    SS_CUDA_B(cudaMemcpyAsync(c->d_tok_row, tok_row.data(), (size_t)T * 4, cudaMemcpyHostToDevice, c->stream));
+    SS_CUDA_B(cudaMemcpyAsync(c->d_tok_pos, tok_pos.data(), (size_t)T * 4, cudaMemcpyHostToDevice, c->stream));
+    SS_CUDA_B(cudaMemcpyAsync(c->d_cu, cu_loc.data(), cu_loc.size() * 4, cudaMemcpyHostToDevice, c->stream));
+    SS_CUDA_B(cudaMemcpyAsync(c->d_last, last.data(), last.size() * 4, cudaMemcpyHostToDevice, c->stream));
+    if ((rc = enqueue_prefill_chunk(c, s0, s1, cu, T))) return bail(rc);
+    SS_CUDA_B(launch(c, gather_last_rmsnorm_kernel, dim3(s1 - s0), dim3(256), 0, (const float*)c->h,
+                     (const int32_t*)c->d_last, c->h_dec + (size_t)s0 * m.d_model, (const bf16*)c->final_norm,
+                     c->x_dec + (size_t)s0 * m.d_model,
+                     (opts && opts->dump_hidden) ? opts->dump_hidden + (size_t)s0 * m.d_model : (float*)nullptr,
+                     m.d_model, m.rms_eps));
+    // the host vectors above are reused by the next chunk
+    SS_CUDA_B(cudaStreamSynchronize(c->stream));
+    s0 = s1;
+  }
+  // LM head on the last tokens, first generated token, bookkeeping
+  const int NT = round_up(B, 16);
+  const CUtensorMap* mx;
+  if ((rc = xmap(c, 3, NT, &mx))) return bail(rc);
+  const GemmPlan p_lm = plan_gemm(m.vocab, m.d_model, NT, 1, kGemmPartial, c->n_sm);
+  if ((rc = run_gemm(c, c->m_lm, *mx, p_lm, kGemmPartial, B, nullptr, nullptr, 0))) return bail(rc);
+  SS_CUDA_B(launch(c, lmhead_argmax_kernel, dim3(B), dim3(1024), 0, (const float*)c->partial, split_of(p_lm), c->st,
+                   opts ? opts->dump_logits : (float*)nullptr, m.vocab, m.eos_id));
+  SS_CUDA_B(launch(c, bookkeeping_kernel, dim3(1), dim3(kMaxBatch), 0, c->st,
+                   opts ? opts->forced_tokens : (const int32_t*)nullptr, first_tokens, B, m.eos_id, 1));
+#undef SS_CUDA_B
+  return SS_OK;
+}
+
+int ss_decode_step(ss_ctx* c, const ss_step_opts* opts, int32_t* next_tokens, int32_t* n_active_host) {
+  if (!c) return SS_ERR_ARG;
+  if (!c->in_batch) return SS_ERR_STATE;
+  int rc = enqueue_decode_step(c, opts, next_tokens);
+  if (rc) return rc;
+  if (n_active_host)
+    SS_CUDA(c, cudaMemcpyAsync(n_active_host, c->st.scalars + 1, 4, cudaMemcpyDeviceToHost, c->stream));
+  return SS_OK;
+}
+
+int ss_decode_steps(ss_ctx* c, int32_t n_steps, int32_t* n_active_host) {
+  if (!c || n_steps < 0) return SS_ERR_ARG;
+  if (!c->in_batch) return SS_ERR_STATE;
+  auto it = c->graphs.find(c->B);
+  if (it == c->graphs.end()) {
+    // make sure every tensor map the step needs exists before capture starts
+    const CUtensorMap* tmp;
+    const int NT = round_up(c->B, 16);
+    int rc;
+    if ((rc = xmap(c, 3, NT, &tmp)) || (rc = xmap(c, 4, NT, &tmp)) || (rc = xmap(c, 5, NT, &tmp))) return rc;
+    cudaGraph_t g = nullptr;
+    SS_CUDA(c, cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
+    c->capturing = true;
+    c->capture_count = 0;
+    rc = enqueue_decode_step(c, nullptr, nullptr);
+    c->capturing = false;
+    cudaError_t e = cudaStreamEndCapture(c->stream, &g);
+    if (rc) { if (g) cudaGraphDestroy(g); return rc; }
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    cudaGraphExec_t ge = nullptr;
+    e = cudaGraphInstantiate(&ge, g, 0);
+    cudaGraphDestroy(g);
+    if (e != cudaSuccess) return cuda_fail(c, e);
+    c->graph_nodes = c->capture_count;
+    it = c->graphs.emplace(c->B, ge).first;
+  }
+  for (int s = 0; s < n_steps; ++s) {
+    SS_CUDA(c, cudaGraphLaunch(it->second, c->stream));
+    c->launches += c->graph_nodes;
+  }
+  if (n_active_host)
+    SS_CUDA(c, cudaMemcpyAsync(n_active_host, c->st.scalars + 1, 4, cudaMemcpyDeviceToHost, c->stream));
+  return SS_OK;
+}
+
+int ss_read_batch(ss_ctx* c, int32_t* out_tokens, int32_t stride, int32_t* out_len, uint8_t* out_status) {
+  if (!c || !out_len || !out_status || (out_tokens && stride < 1)) return SS_ERR_ARG;
+  if (!c->in_batch) return SS_ERR_STATE;
+  const int B = c->B;
+  std::vector<int32_t> gen(B), fin(B);
+  SS_CUDA(c, cudaMemcpyAsync(gen.data(), c->st.gen, (size_t)B * 4, cudaMemcpyDeviceToHost, c->stream));
+  SS_CUDA(c, cudaMemcpyAsync(fin.data(), c->st.finished, (size_t)B * 4, cudaMemcpyDeviceToHost, c->stream));
+  SS_CUDA(c, cudaMemcpyAsync(c->pinned + 1, c->status, 4, cudaMemcpyDeviceToHost, c->stream));
+  SS_CUDA(c, cudaStreamSynchronize(c->stream));
+  if (c->pinned[1] != 0) return c->pinned[1] == (int32_t)kStatusBadPage ? SS_ERR_STATE : SS_ERR_DEVICE_TIMEOUT;
+  for (int r = 0; r < B; ++r) {
+    if (out_tokens && gen[r] > stride) return SS_ERR_CAPACITY;
+    out_len[r] = gen[r];
+    out_status[r] = fin[r] ? 1 : 0;
+  }
+  if (out_tokens) {
+    for (int r = 0; r < B; ++r)
+      if (gen[r] > 0)
+        SS_CUDA(c, cudaMemcpyAsync(out_tokens + (size_t)r * stride, c->st.out_tokens + (size_t)r * c->st.max_new,
+                                   (size_t)gen[r] * 4, cudaMemcpyDeviceToHost, c->stream));
+    SS_CUDA(c, cudaStreamSynchronize(c->stream));
+  }
+  return SS_OK;
+}
+
+int ss_step_model_bytes(const ss_ctx* c, const int32_t* ctx_len, const uint8_t* active, int32_t B, double* out) {
+  if (!c || !ctx_len || !out || B < 0) return SS_ERR_ARG;
+  double bytes = weight_bytes_per_step(c->m);
+  const double kvt = kv_bytes_per_token(c->m);
+  for (int r = 0; r < B; ++r)
+    if (!active || active[r]) bytes += kvt * ((double)ctx_len[r] + 1.0) + (double)c->m.d_model * 2.0;
+  *out = bytes;
+  return SS_OK;
+}
+
+int ss_last_device_status(ss_ctx* c, uint32_t* out) {
+  if (!c || !out) return SS_ERR_ARG;
+  SS_CUDA(c, cudaMemcpyAsync(c->pinned + 1, c->status, 4, cudaMemcpyDeviceToHost, c->stream));
+  SS_CUDA(c, cudaStreamSynchronize(c->stream));
+  *out = (uint32_t)c->pinned[1];
+  return SS_OK;
+}
+
+int ss_last_cuda_error(const ss_ctx* c) { return c ? c->last_cuda : 0; }
+int64_t ss_kernel_launches(const ss_ctx* c) { return c ? c->launches : 0; }
+
+int ss_run_group(ss_ctx* c, const ss_sched_cfg* cfg, const int32_t* prompt_tokens, const int64_t* prompt_off,
+                 const int32_t* pred_len, const int32_t* perm, const int32_t* eos_at, int32_t n, int32_t* out_tokens,
+                 const int64_t* out_off, int32_t* out_len, uint8_t* out_status, int32_t* order, ss_batch_log* log,
+                 int32_t log_cap, int32_t* n_log, ss_group_stats* stats) {
+  if (!c || !cfg || n < 0 || !n_log) return SS_ERR_ARG;
+  if (n > 0 && (!prompt_tokens || !prompt_off || !pred_len || !out_tokens || !out_off || !out_len || !out_status || !order))
+    return SS_ERR_ARG;
+  int rc = validate_sched_cfg(cfg);
+  if (rc) return rc;
+  if (c->in_batch) return SS_ERR_STATE;
+  if (cfg->max_new_tokens > c->rt.max_new_tokens) return SS_ERR_CAPACITY;
+  for (int i = 0; i < n; ++i)
+    if (out_off[i + 1] - out_off[i] < cfg->max_new_tokens) return SS_ERR_CAPACITY;
+
+  std::vector<int32_t> plen(n);
+  for (int i = 0; i < n; ++i) plen[i] = (int32_t)(prompt_off[i + 1] - prompt_off[i]);
+  std::vector<int32_t> ord;
+  std::vector<ss_batch_desc> plan;
+  if ((rc = plan_first_pass(*cfg, plen.data(), pred_len, perm, n, ord, plan))) return rc;
+  std::copy(ord.begin(), ord.end(), order);
+
+  cudaEvent_t ev[3];
+  for (auto& e : ev) SS_CUDA(c, cudaEventCreate(&e));
+  auto destroy_events = [&]() { for (auto& e : ev) cudaEventDestroy(e); };
+
+  ss_group_stats gs{};
+  const int64_t launches0 = c->launches;
+  const double W = weight_bytes_per_step(c->m), kvt = kv_bytes_per_token(c->m);
+  std::vector<int32_t> fail_rows;
+  std::vector<int32_t> toks, cu, eos_b, len_b;
+  std::vector<uint8_t> st_b;
+  std::vector<int32_t> tok_b;
+  int n_batches = 0;
+  size_t next_fail = 0;
+  size_t bi = 0;
+  const int B0 = cfg->base_batch;
+  cudaEvent_t g0, g1;
+  SS_CUDA(c, cudaEventCreate(&g0));
+  SS_CUDA(c, cudaEventCreate(&g1));
+  SS_CUDA(c, cudaEventRecord(g0, c->stream));
+  auto cleanup = [&](int code) {
+    destroy_events();
+    cudaEventDestroy(g0);
+    cudaEventDestroy(g1);
+    if (c->in_batch) ss_release_batch(c);
+    return code;
+  };
+  for (;;) {
+    ss_batch_desc b;
+    const int32_t* rows_src;
+    if (bi < plan.size()) {
+      b = plan[bi++];
+      rows_src = ord.data() + b.first_row;
+    } else if (next_fail < fail_rows.size()) {
+      const int nr = (int)std::min<size_t>(B0, fail_rows.size() - next_fail);
+      b = {(int32_t)(n + next_fail), nr, cfg->max_new_tokens, 1};
+      rows_src = fail_rows.data() + next_fail;
+      next_fail += nr;
+    } else {
+      break;
+    }
+    const int B = b.n_rows;
+    if (n_batches >= log_cap && log) return cleanup(SS_ERR_CAPACITY);
+    toks.clear();
+    cu.assign(1, 0);
+    eos_b.clear();
+    int max_target = 0;
+    for (int r = 0; r < B; ++r) {
+      const int q = rows_src[r];
+      toks.insert(toks.end(), prompt_tokens + prompt_off[q], prompt_tokens + prompt_off[q + 1]);
+      cu.push_back((int32_t)toks.size());
+      if (eos_at) { eos_b.push_back(eos_at[q]); max_target = std::max(max_target, eos_at[q]); }
+    }
+    SS_CUDA(c, cudaEventRecord(ev[0], c->stream));
+    rc = ss_prefill(c, toks.data(), cu.data(), B, eos_at ? eos_b.data() : nullptr, b.cap, nullptr, nullptr);
+    if (rc) return cleanup(rc);
+    SS_CUDA(c, cudaEventRecord(ev[1], c->stream));
+    if (eos_at) {
+      // lengths are forced, so the number of steps is known: the longest target or the cap
+      const int steps = std::min(b.cap, max_target);
+      if ((rc = ss_decode_steps(c, steps - 1, nullptr))) return cleanup(rc);
+    } else {
+      int done = 1;
+      while (done < b.cap) {
+        const int chunk = std::min(8, b.cap - done);
+        if ((rc = ss_decode_steps(c, chunk, c->pinned))) return cleanup(rc);
+        SS_CUDA(c, cudaStreamSynchronize(c->stream));
+        done += chunk;
+        if (c->pinned[0] == 0) break;
+      }
+    }
+    SS_CUDA(c, cudaEventRecord(ev[2], c->stream));
+    len_b.assign(B, 0);
+    st_b.assign(B, 0);
+    tok_b.assign((size_t)B * cfg->max_new_tokens, 0);
+    if ((rc = ss_read_batch(c, tok_b.data(), cfg->max_new_tokens, len_b.data(), st_b.data()))) return cleanup(rc);
+    ss_release_batch(c);
+    float pf = 0, dc = 0;
+    cudaEventElapsedTime(&pf, ev[0], ev[1]);
+    cudaEventElapsedTime(&dc, ev[1], ev[2]);
+    int steps = 0, n_failed = 0;
+    for (int r = 0; r < B; ++r) {
+      const int q = rows_src[r];
+      steps = std::max(steps, len_b[r]);
+      const bool failed = !st_b[r] && b.cap < cfg->max_new_tokens;
+      if (failed) {
+        fail_rows.push_back(q);
+        ++n_failed;
+      } else {
+        out_len[q] = len_b[r];
+        out_status[q] = st_b[r];
+        std::copy(tok_b.begin() + (size_t)r * cfg->max_new_tokens,
+                  tok_b.begin() + (size_t)r * cfg->max_new_tokens + len_b[r], out_tokens + out_off[q]);
+        gs.useful_tokens += len_b[r];
+      }
+      const double nr = std::max(0, len_b[r] - 1);     // decode steps the row took part in
+      gs.model_bytes += kvt * (nr * (cu[r + 1] - cu[r]) + nr * (nr + 1) / 2.0);
+    }
+    gs.model_bytes += W * std::max(0, steps - 1);
+    if (log) log[n_batches] = {b.first_row, B, b.cap, b.is_recompute, steps, n_failed, pf, dc};
+    ++n_batches;
+    gs.steps += steps;
+    gs.row_steps += (int64_t)B * steps;
+    gs.prefill_ms += pf;
+    gs.decode_ms += dc;
+    gs.n_failed += n_failed;
+  }
+  for (size_t i = 0; i < fail_rows.size(); ++i) order[n + i] = fail_rows[i];
+  for (size_t i = fail_rows.size(); i < (size_t)n; ++i) order[n + i] = -1;
+  SS_CUDA(c, cudaEventRecord(g1, c->stream));
+  SS_CUDA(c, cudaEventSynchronize(g1));
+  cudaEventElapsedTime(&gs.total_ms, g0, g1);
+  gs.n_batches = n_batches;
+  gs.kernel_launches = c->launches - launches0;
+  *n_log = n_batches;
+  if (stats) *stats = gs;
+  return cleanup(SS_OK);
+}
+
+}  // extern "C"
