@@ -123,8 +123,10 @@ typedef struct {
 int ss_arena_bytes(const ss_model_cfg* model, const ss_runtime_cfg* rt, size_t* out_bytes);
 
 /* Creates a context.  dev_arena: device memory, 1024-byte aligned, at least ss_arena_bytes().
- * It must outlive the context.  stream: cudaStream_t.  SS_ERR_UNSUPPORTED for shapes the
- * kernels do not cover, SS_ERR_CAPACITY for a short arena. */
+ * It must outlive the context.  stream: cudaStream_t; ss_decode_steps() and ss_run_group()
+ * capture CUDA graphs on it, which the legacy default stream (0) does not allow, so pass a
+ * stream created by the caller.  SS_ERR_UNSUPPORTED for shapes the kernels do not cover,
+ * SS_ERR_CAPACITY for a short arena. */
 int ss_create(const ss_model_cfg* model, const ss_runtime_cfg* rt, void* dev_arena, size_t arena_bytes,
               void* stream, ss_ctx** out);
 int ss_destroy(ss_ctx* ctx);

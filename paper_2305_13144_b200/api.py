@@ -111,8 +111,10 @@ def ss_strerror(code: int) -> str:
     return lib().ss_strerror(int(code)).decode()
 
 
-def _check(code: int, where: str) -> None:
+def _check(code: int, where: str, ctx=None) -> None:
     if code != SS_OK:
+        if code == SS_ERR_CUDA and ctx is not None and ctx.handle:
+            where += f" [cuda error {lib().ss_last_cuda_error(ctx.handle)}]"
         raise SSError(code, where)
 
 
@@ -203,7 +205,7 @@ def ss_load_weights(ctx: Ctx, tensors: dict) -> None:
             ptr, dev, shape = t.data_ptr(), int(t.is_cuda), tuple(t.shape)
         rows, cols = (1, shape[0]) if len(shape) == 1 else shape
         descs[i] = ss_tensor_desc(name.encode(), ptr, dev, rows, cols)
-    _check(lib().ss_load_weights(ctx.handle, descs, len(tensors)), "ss_load_weights")
+    _check(lib().ss_load_weights(ctx.handle, descs, len(tensors)), "ss_load_weights", ctx)
 
 
 def ss_schedule(cfg: ss_sched_cfg, prompt_len, pred_len, perm=None):
@@ -230,7 +232,7 @@ def ss_prefill(ctx: Ctx, tokens, cu_seqlens, eos_at, cap: int, *, forced_tokens=
     tk, cu, ea = _np(tokens, np.int32), _np(cu_seqlens, np.int32), _np(eos_at, np.int32)
     o = _opts(forced_tokens, dump_logits, dump_hidden)
     _check(lib().ss_prefill(ctx.handle, _hp(tk), _hp(cu), int(cu.shape[0]) - 1, _hp(ea), int(cap),
-                            C.byref(o) if o else None, _dp(first_tokens)), "ss_prefill")
+                            C.byref(o) if o else None, _dp(first_tokens)), "ss_prefill", ctx)
 
 
 def ss_decode_step(ctx: Ctx, *, forced_tokens=None, dump_logits=None, dump_hidden=None, next_tokens=None,
@@ -238,24 +240,24 @@ def ss_decode_step(ctx: Ctx, *, forced_tokens=None, dump_logits=None, dump_hidde
     """n_active_host: pinned int32 torch tensor (host) or None."""
     o = _opts(forced_tokens, dump_logits, dump_hidden)
     nah = None if n_active_host is None else C.c_void_p(n_active_host.data_ptr())
-    _check(lib().ss_decode_step(ctx.handle, C.byref(o) if o else None, _dp(next_tokens), nah), "ss_decode_step")
+    _check(lib().ss_decode_step(ctx.handle, C.byref(o) if o else None, _dp(next_tokens), nah), "ss_decode_step", ctx)
 
 
 def ss_decode_steps(ctx: Ctx, n_steps: int, n_active_host=None) -> None:
     nah = None if n_active_host is None else C.c_void_p(n_active_host.data_ptr())
-    _check(lib().ss_decode_steps(ctx.handle, int(n_steps), nah), "ss_decode_steps")
+    _check(lib().ss_decode_steps(ctx.handle, int(n_steps), nah), "ss_decode_steps", ctx)
 
 
 def ss_read_batch(ctx: Ctx, B: int, stride: int):
     toks = np.zeros((B, stride), dtype=np.int32)
     lens = np.zeros(B, dtype=np.int32)
     status = np.zeros(B, dtype=np.uint8)
-    _check(lib().ss_read_batch(ctx.handle, _hp(toks), stride, _hp(lens), _hp(status)), "ss_read_batch")
+    _check(lib().ss_read_batch(ctx.handle, _hp(toks), stride, _hp(lens), _hp(status)), "ss_read_batch", ctx)
     return toks, lens, status
 
 
 def ss_release_batch(ctx: Ctx) -> None:
-    _check(lib().ss_release_batch(ctx.handle), "ss_release_batch")
+    _check(lib().ss_release_batch(ctx.handle), "ss_release_batch", ctx)
 
 
 def ss_run_group(ctx: Ctx, cfg: ss_sched_cfg, prompt_tokens, prompt_off, pred_len, perm=None, eos_at=None) -> dict:
@@ -274,7 +276,7 @@ def ss_run_group(ctx: Ctx, cfg: ss_sched_cfg, prompt_tokens, prompt_off, pred_le
     stats = ss_group_stats()
     _check(lib().ss_run_group(ctx.handle, C.byref(cfg), _hp(pt), _hp(po), _hp(pr), _hp(pm), _hp(ea), n,
                               _hp(out_tokens), _hp(out_off), _hp(out_len), _hp(out_status), _hp(order),
-                              log, log_cap, C.byref(n_log), C.byref(stats)), "ss_run_group")
+                              log, log_cap, C.byref(n_log), C.byref(stats)), "ss_run_group", ctx)
     fields = [f[0] for f in ss_batch_log._fields_]
     return {
         "tokens": out_tokens.reshape(n, mx) if n else out_tokens[:0].reshape(0, mx),
@@ -294,7 +296,7 @@ def ss_step_model_bytes(ctx: Ctx, ctx_len, active=None) -> float:
 
 def ss_last_device_status(ctx: Ctx) -> int:
     out = C.c_uint32(0)
-    _check(lib().ss_last_device_status(ctx.handle, C.byref(out)), "ss_last_device_status")
+    _check(lib().ss_last_device_status(ctx.handle, C.byref(out)), "ss_last_device_status", ctx)
     return out.value
 
 
@@ -311,12 +313,17 @@ def runtime_cfg(max_batch, max_ctx, max_prefill_tokens, max_new_tokens, kv_pool_
 
 
 def make_engine(shape, rt: ss_runtime_cfg, weights: dict, device="cuda:0") -> Ctx:
-    """Convenience for tests and the benchmark: allocate the arena with torch, create, load weights."""
+    """Convenience for tests and the benchmark: allocate the arena with torch, create, load weights.
+
+    The engine gets a stream of its own: CUDA graphs (ss_decode_steps, ss_run_group) cannot be
+    captured on the legacy default stream.  Callers order their own work against it with
+    torch.cuda.synchronize() or stream events."""
     import torch
     m = model_cfg(shape)
     nbytes = ss_arena_bytes(m, rt)
     with torch.cuda.device(device):
         arena = torch.empty(nbytes + 1024, dtype=torch.uint8, device=device)
-        ctx = ss_create(m, rt, arena)
+        torch.cuda.synchronize()
+        ctx = ss_create(m, rt, arena, torch.cuda.Stream())
         ss_load_weights(ctx, weights)
     return ctx

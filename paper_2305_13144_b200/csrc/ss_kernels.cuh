@@ -232,7 +232,9 @@ __global__ void __launch_bounds__(128) attn_decode_kernel(AttnArgs a) {
     for (int j = 0; j < 8; ++j) acc[j] = 0.f;
 
     constexpr int U = 4;
-    for (int tb = t0 + g; tb < t1; tb += NG * U) {
+    // the trip count is the same for every lane of the warp (the shuffles below need all of them)
+    for (int base = t0; base < t1; base += NG * U) {
+      const int tb = base + g;
       uint4 kk[U], vv[U];
       bool valid[U];
 #pragma unroll
