@@ -265,7 +265,8 @@ __global__ void __launch_bounds__(128) attn_decode_kernel(AttnArgs a) {
       float mn = m;
 #pragma unroll
       for (int u = 0; u < U; ++u) mn = fmaxf(mn, s[u]);
-      const float sc = exp2f(m - mn);           // m = -inf on the first pass -> 0
+      // a group that has seen no key yet keeps (m, l, acc) = (-inf, 0, 0): exp2(-inf - -inf) would be NaN
+      const float sc = (mn == -CUDART_INF_F) ? 1.f : exp2f(m - mn);
       l *= sc;
 #pragma unroll
       for (int j = 0; j < 8; ++j) acc[j] *= sc;

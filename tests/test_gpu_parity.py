@@ -101,6 +101,16 @@ def test_tiny_ragged_batch_sizes_and_page_boundaries():
         assert el <= LOGIT_TOL and eh <= HIDDEN_TOL, (B, el, eh)
 
 
+def test_very_short_prompts_leave_attention_groups_without_keys():
+    """Fewer cached tokens than key groups in the decode-attention CTA (prompts of 1, 2, 5 tokens)."""
+    shape = synth.TINY
+    w = synth.make_weights(shape, seed=1234)
+    rng = np.random.default_rng(11)
+    prompts = [rng.integers(3, shape.vocab, size=n).tolist() for n in (1, 2, 5, 9, 14, 30)]
+    el, eh = _teacher_forced(shape, w, prompts, [6, 6, 5, 4, 6, 3], cap=6)
+    assert el <= LOGIT_TOL and eh <= HIDDEN_TOL, (el, eh)
+
+
 def test_long_context_spans_attention_chunks():
     """A prompt longer than one attention work item (256 tokens) and one prompt-pass query tile."""
     shape = synth.TINY.with_layers(1)
