@@ -209,6 +209,29 @@ int ss_run_group(ss_ctx* ctx, const ss_sched_cfg* cfg, const int32_t* prompt_tok
  * ctx_len host [B] (tokens cached before the step), active host uint8 [B]. */
 int ss_step_model_bytes(const ss_ctx* ctx, const int32_t* ctx_len, const uint8_t* active, int32_t B, double* out);
 
+/* (The paper has no counterpart to this call; it exists for integration.)
+ * The LM-head projection for callers that cannot allocate device memory: code running while
+ * its framework captures a CUDA graph, inside an allocator callback, in a process whose device
+ * memory is all handed to another pool, or in a loop where an allocation's hidden
+ * synchronisation is not acceptable.  Computes, with the same kernels as the engine,
+ *     logits[r][v] = sum_i lm_head[v][i] * bf16( hidden[r][i] * rsqrt(mean_j hidden[r][j]^2 + eps) * gain[i] )
+ *   hidden    device fp32 [n_rows, d_model]      norm_gain device bf16 [d_model]
+ *   lm_head   device bf16 [vocab, d_model], 16-byte aligned
+ *   logits    device fp32 [n_rows, vocab] (output)      stream  cudaStream_t
+ * No ss_ctx, no arena: the two temporaries (bf16 activations, fp32 split-K partial sums) live in
+ * an 8 MiB array that is part of the library image, so every GPU that loads the library holds
+ * those 8 MiB until the process ends.  The call itself allocates nothing on the device or the
+ * host.  Limits: n_rows <= 16, d_model <= 8192 and a multiple of 64, and vocab small enough for
+ * the partial sums to fit (vocab 32000 uses 3.7 MiB; on a 148-SM part a vocab of about 94000 is
+ * the edge); beyond them SS_ERR_CAPACITY is returned and nothing is launched.
+ * The first call on each device looks up the array's device address and raises the kernel's
+ * shared-memory limit; make that first call, with the device current, before any stream capture.
+ * All calls share the one array and it keeps what the last call left there (the call clears the
+ * only word that must start at zero), so two calls whose kernels may overlap on the GPU --
+ * different streams, or threads -- race; keep calls on one device in one stream order. */
+int ss_logits_noalloc(const float* hidden, const void* norm_gain, const void* lm_head, int32_t n_rows,
+                      int32_t d_model, int32_t vocab, float rms_eps, float* logits, void* stream);
+
 const char* ss_strerror(int code);
 /* Last device status word (0 = clean; non-zero = which bounded wait expired). Synchronises. */
 int ss_last_device_status(ss_ctx* ctx, uint32_t* out);

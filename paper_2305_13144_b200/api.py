@@ -23,6 +23,7 @@ EXPORTS = [
     "ss_arena_bytes", "ss_create", "ss_destroy", "ss_load_weights", "ss_schedule", "ss_prefill",
     "ss_decode_step", "ss_decode_steps", "ss_read_batch", "ss_release_batch", "ss_run_group",
     "ss_step_model_bytes", "ss_strerror", "ss_last_device_status", "ss_last_cuda_error", "ss_kernel_launches",
+    "ss_logits_noalloc",
 ]
 
 
@@ -103,6 +104,8 @@ def lib() -> C.CDLL:
         L.ss_run_group.argtypes = [C.c_void_p] * 7 + [C.c_int32] + [C.c_void_p] * 6 + [C.c_int32, C.c_void_p, C.c_void_p]
         L.ss_step_model_bytes.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(C.c_double)]
         L.ss_last_device_status.argtypes = [C.c_void_p, C.POINTER(C.c_uint32)]
+        L.ss_logits_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
+                                        C.c_float, C.c_void_p, C.c_void_p]
         _lib_handle = L
     return _lib_handle
 
@@ -306,6 +309,24 @@ def ss_last_cuda_error(ctx: Ctx) -> int:
 
 def ss_kernel_launches(ctx: Ctx) -> int:
     return lib().ss_kernel_launches(ctx.handle)
+
+
+def ss_logits_noalloc(hidden, norm_gain, lm_head, rms_eps: float, logits, stream=None) -> None:
+    """LM-head logits without any allocation by the library (see include/seqsched.h).
+
+    hidden fp32 [n, d], norm_gain bf16 [d], lm_head bf16 [V, d], logits fp32 [n, V]: CUDA tensors
+    the caller made beforehand.  Scratch comes from a fixed array inside the library, shared by
+    all calls: keep the calls of one device in one stream order."""
+    import torch
+    n, d = hidden.shape
+    V = lm_head.shape[0]
+    if hidden.dtype != torch.float32 or logits.dtype != torch.float32 or tuple(logits.shape) != (n, V):
+        raise ValueError("hidden and logits must be fp32 [n, d] / [n, V]")
+    if norm_gain.element_size() != 2 or lm_head.element_size() != 2:
+        raise ValueError("norm_gain and lm_head must be bf16")
+    st = torch.cuda.current_stream() if stream is None else stream
+    _check(lib().ss_logits_noalloc(_dp(hidden), _dp(norm_gain), _dp(lm_head), n, d, V, float(rms_eps), _dp(logits),
+                                   C.c_void_p(st.cuda_stream)), "ss_logits_noalloc")
 
 
 def runtime_cfg(max_batch, max_ctx, max_prefill_tokens, max_new_tokens, kv_pool_tokens) -> ss_runtime_cfg:

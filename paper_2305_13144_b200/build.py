@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libseqsched.so")
-SOURCES = ["ss_runtime.cu", "ss_sched.cpp"]
+SOURCES = ["ss_runtime.cu", "ss_noalloc.cu", "ss_sched.cpp"]
 HEADERS = ["ss_internal.h", "ss_gemm.cuh", "ss_kernels.cuh"]
 
 

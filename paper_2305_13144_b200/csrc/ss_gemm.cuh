@@ -168,7 +168,8 @@ struct GemmSmemHeader {
   uint32_t pad;
 };
 
-__global__ void __launch_bounds__(kGemmThreads, 1)
+// internal linkage: the header is compiled into more than one translation unit
+static __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_wx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, GemmArgs a) {
   extern __shared__ uint8_t smem_raw[];
   const GemmPlan& p = a.p;
