@@ -141,8 +141,9 @@ __host__ __device__ __forceinline__ int split_owner(const SplitInfo& s, long lon
   while (c + 1 < s.gridx && split_begin(s, c + 1) <= x) ++c;
   return c;
 }
-// Sum of the fp32 partials of output row n (of n_out) for token `tok`, in CTA order.
-__device__ __forceinline__ float sum_partials(const float* __restrict__ partial, const SplitInfo& s, int n, int tok) {
+// Sum of the fp32 partials of output row n (of n_out) for token `tok`, in CTA order; the tile's
+// segments are derived from the split arithmetic on the fly (several 64-bit divisions).
+__device__ __forceinline__ float sum_partials_derived(const float* __restrict__ partial, const SplitInfo& s, int n, int tok) {
   const int tile = n >> 7, row = n & 127;
   const long long x0 = (long long)tile * s.kb;
   const int c0 = split_owner(s, x0), c1 = split_owner(s, x0 + s.kb - 1);
@@ -152,6 +153,16 @@ __device__ __forceinline__ float sum_partials(const float* __restrict__ partial,
     const size_t slot = (size_t)c * s.max_seg + seg;
     acc += partial[(slot * s.NT + tok) * 128 + row];
   }
+  return acc;
+}
+// The same sum with the tile's segments read from the precomputed table (same order, same bits).
+__device__ __forceinline__ float sum_partials(const float* __restrict__ partial, const SplitInfo& s, int n, int tok) {
+  const int4 t = __ldg(reinterpret_cast<const int4*>(s.tiles) + (n >> 7));
+  const size_t slot_stride = (size_t)s.NT * 128;
+  const size_t off = (size_t)tok * 128 + (n & 127);
+  float acc = partial[(size_t)t.x * slot_stride + off];
+  const size_t cta_stride = slot_stride * s.max_seg;
+  for (int c = t.y; c <= t.z; ++c) acc += partial[(size_t)c * cta_stride + off];
   return acc;
 }
 

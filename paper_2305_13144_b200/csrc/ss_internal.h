@@ -61,10 +61,17 @@ struct GemmArgs {
   uint32_t* status;
 };
 
+// Where the partial sums of one 128-row tile live: the first segment in slot `slot0`, the others
+// in segment 0 of CTAs c_next..c_last (a CTA that starts inside a tile has it as its first tile).
+struct TileSeg {
+  int32_t slot0, c_next, c_last, pad;
+};
+
 // Partial-slot bookkeeping shared by the GEMM and its consumers.
 struct SplitInfo {
   int gridx, kb, max_seg, NT;
-  long long total;     // n_tiles * kb
+  long long total;          // n_tiles * kb
+  const TileSeg* tiles;     // device table [n_tiles], or null (then the consumers derive it)
 };
 
 }  // namespace ss

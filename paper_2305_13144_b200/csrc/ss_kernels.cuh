@@ -89,25 +89,32 @@ embed_rmsnorm_kernel(const int32_t* __restrict__ tokens, const int32_t* __restri
 }
 
 // ------------------------------------------------------------------------------------ RoPE + KV append (decode)
-// grid (H, B), block Dh/2.  q,k,v come as fp32 partials of the [3d] projection.
-// Pair (i, i+Dh/2) of q and k is rotated by pos * inv_freq[i]; k,v go to the row's page.
-__global__ void rope_append_decode_kernel(const float* __restrict__ partial, SplitInfo sp, RowState st, KvLayout kv,
-                                          int layer, const float* __restrict__ inv_freq, bf16* __restrict__ qbuf,
-                                          int d, uint32_t* status) {
+// grid (H, B), block Dh.  q,k,v come as fp32 partials of the [3d] projection; thread i owns element
+// i of the head.  Pair (i, i+Dh/2) of q and k is rotated by pos * inv_freq[i]; k,v go to the row's page.
+__global__ void __launch_bounds__(128)
+rope_append_decode_kernel(const float* __restrict__ partial, SplitInfo sp, RowState st, KvLayout kv, int layer,
+                          const float* __restrict__ inv_freq, bf16* __restrict__ qbuf, int d, uint32_t* status) {
+  __shared__ float s_q[128], s_k[128];
   pdl_launch_dependents();
   pdl_wait();
   const int hd = blockIdx.x, r = blockIdx.y, i = threadIdx.x;
   if (!st.active[r]) return;
   const int Dh = kv.Dh, half = Dh >> 1;
   const int pos = st.ctx_len[r];
-  const int n0 = hd * Dh + i, n1 = n0 + half;
-  const float q0 = sum_partials(partial, sp, n0, r), q1 = sum_partials(partial, sp, n1, r);
-  const float k0 = sum_partials(partial, sp, d + n0, r), k1 = sum_partials(partial, sp, d + n1, r);
-  const float v0 = sum_partials(partial, sp, 2 * d + n0, r), v1 = sum_partials(partial, sp, 2 * d + n1, r);
+  const int n = hd * Dh + i;
+  const float qv = sum_partials(partial, sp, n, r);
+  const float kvv = sum_partials(partial, sp, d + n, r);
+  const float vv = sum_partials(partial, sp, 2 * d + n, r);
+  s_q[i] = qv;
+  s_k[i] = kvv;
+  __syncthreads();
+  const int j = i < half ? i : i - half;          // frequency index
   float sn, cs;
-  sincosf((float)pos * inv_freq[i], &sn, &cs);
-  qbuf[(size_t)r * d + n0] = __float2bfloat16_rn(q0 * cs - q1 * sn);
-  qbuf[(size_t)r * d + n1] = __float2bfloat16_rn(q1 * cs + q0 * sn);
+  sincosf((float)pos * inv_freq[j], &sn, &cs);
+  // first half: x_i cos - x_{i+half} sin; second half: x_i cos + x_{i-half} sin
+  const float qo = i < half ? qv * cs - s_q[i + half] * sn : qv * cs + s_q[i - half] * sn;
+  const float ko = i < half ? kvv * cs - s_k[i + half] * sn : kvv * cs + s_k[i - half] * sn;
+  qbuf[(size_t)r * d + n] = __float2bfloat16_rn(qo);
   const int page = st.block_table[(size_t)r * st.max_pages + pos / kPageTokens];
   if (page < 0 || page >= kv.n_pages) {
     atomicCAS(status, 0u, (uint32_t)kStatusBadPage);
@@ -116,10 +123,8 @@ __global__ void rope_append_decode_kernel(const float* __restrict__ partial, Spl
   bf16* kbase = kv.pool + (size_t)layer * kv.layer_stride + (size_t)page * kv.page_elems +
                 ((size_t)hd * kPageTokens + (pos % kPageTokens)) * Dh;
   bf16* vbase = kbase + (size_t)kv.H * kPageTokens * Dh;
-  kbase[i] = __float2bfloat16_rn(k0 * cs - k1 * sn);
-  kbase[i + half] = __float2bfloat16_rn(k1 * cs + k0 * sn);
-  vbase[i] = __float2bfloat16_rn(v0);
-  vbase[i + half] = __float2bfloat16_rn(v1);
+  kbase[i] = __float2bfloat16_rn(ko);
+  vbase[i] = __float2bfloat16_rn(vv);
 }
 
 // ------------------------------------------------------------------------------------ decode attention (paged)
@@ -328,8 +333,8 @@ __global__ void __launch_bounds__(DH) attn_combine_kernel(AttnArgs a) {
 }
 
 // ------------------------------------------------------------------------------------ residual + RMSNorm (decode)
-// h[r] += projection (from partials); x[r] = RMSNorm(h[r]) * g.  grid B, block 256.
-__global__ void __launch_bounds__(256)
+// h[r] += projection (from partials); x[r] = RMSNorm(h[r]) * g.  grid B, block 1024 (d <= 8192).
+__global__ void __launch_bounds__(1024)
 residual_rmsnorm_partial_kernel(const float* __restrict__ partial, SplitInfo sp, const int32_t* __restrict__ active,
                                 float* __restrict__ h, const bf16* __restrict__ g, bf16* __restrict__ x,
                                 float* __restrict__ dump_hidden, int d, float eps) {
@@ -338,12 +343,12 @@ residual_rmsnorm_partial_kernel(const float* __restrict__ partial, SplitInfo sp,
   pdl_wait();
   const int r = blockIdx.x;
   if (active && !active[r]) return;
-  constexpr int kMaxPer = 32;                      // d <= 8192
+  constexpr int kMaxPer = 8;
   float v[kMaxPer];
   float ss = 0.f;
 #pragma unroll
   for (int c = 0; c < kMaxPer; ++c) {
-    const int i = threadIdx.x + c * 256;
+    const int i = threadIdx.x + c * 1024;
     v[c] = 0.f;
     if (i < d) {
       v[c] = h[(size_t)r * d + i] + sum_partials(partial, sp, i, r);
@@ -354,7 +359,7 @@ residual_rmsnorm_partial_kernel(const float* __restrict__ partial, SplitInfo sp,
   const float inv = rsqrtf(ss / d + eps);
 #pragma unroll
   for (int c = 0; c < kMaxPer; ++c) {
-    const int i = threadIdx.x + c * 256;
+    const int i = threadIdx.x + c * 1024;
     if (i < d) {
       h[(size_t)r * d + i] = v[c];
       if (dump_hidden) dump_hidden[(size_t)r * d + i] = v[c];
@@ -376,78 +381,105 @@ swiglu_partial_kernel(const float* __restrict__ partial, SplitInfo sp, bf16* __r
 }
 
 // ------------------------------------------------------------------------------------ LM head argmax
-// grid B, block 1024: logits from partials, optional dump, argmax with lowest id on ties,
-// EOS left out when the row has a forced-EOS schedule.
-__global__ void __launch_bounds__(1024)
-lmhead_argmax_kernel(const float* __restrict__ partial, SplitInfo sp, RowState st, float* __restrict__ dump_logits,
-                     int vocab, int eos_id) {
-  __shared__ float s_v[32];
-  __shared__ int s_i[32];
+// Stage 1, grid n_tiles (of the vocabulary), block 128 (thread = vocabulary row of the tile):
+// logits from partials for every row of the batch, optional dump, and the tile's best (value, id)
+// per batch row; the lowest id wins a tie; EOS is left out when the row has a forced-EOS schedule.
+// Stage 2 (inside bookkeeping_kernel) picks the best tile per row.
+__device__ __forceinline__ uint32_t float_order_key(float f) {      // monotone float -> uint32
+  const uint32_t u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+__global__ void __launch_bounds__(128)
+lmhead_tile_argmax_kernel(const float* __restrict__ partial, SplitInfo sp, RowState st, float* __restrict__ dump_logits,
+                          float* __restrict__ tile_val, int32_t* __restrict__ tile_idx, int B, int vocab, int n_tiles,
+                          int eos_id) {
+  __shared__ uint32_t s_key[4][kMaxBatch];
+  __shared__ int s_id[4][kMaxBatch];
   pdl_launch_dependents();
   pdl_wait();
-  const int r = blockIdx.x;
-  if (!st.active[r]) return;
-  const bool suppress = st.eos_at[r] > 0;
-  float best = -CUDART_INF_F;
-  int bi = 0x7fffffff;
-  for (int v = threadIdx.x; v < vocab; v += blockDim.x) {
-    const float lg = sum_partials(partial, sp, v, r);
-    if (dump_logits) dump_logits[(size_t)r * vocab + v] = lg;
-    if (suppress && v == eos_id) continue;
-    if (lg > best) { best = lg; bi = v; }       // ascending v: strict '>' keeps the lowest id
-  }
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    const float ov = __shfl_xor_sync(0xffffffffu, best, o);
-    const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-    if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
-  }
-  if (lane == 0) { s_v[warp] = best; s_i[warp] = bi; }
-  __syncthreads();
-  if (warp == 0) {
-    best = s_v[lane];
-    bi = s_i[lane];
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const float ov = __shfl_xor_sync(0xffffffffu, best, o);
-      const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-      if (ov > best || (ov == best && oi < bi)) { best = ov; bi = oi; }
+  const int tile = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int v = tile * 128 + threadIdx.x;
+  for (int r = 0; r < B; ++r) {
+    uint32_t key = 0;                              // below every real key
+    if (st.active[r]) {
+      if (v < vocab) {
+        const float lg = sum_partials(partial, sp, v, r);
+        if (dump_logits) dump_logits[(size_t)r * vocab + v] = lg;
+        if (!(st.eos_at[r] > 0 && v == eos_id)) key = float_order_key(lg);
+      }
+      const uint32_t best = __reduce_max_sync(0xffffffffu, key);
+      const uint32_t who = __ballot_sync(0xffffffffu, key == best);
+      if (lane == 0) {
+        s_key[warp][r] = best;
+        s_id[warp][r] = tile * 128 + warp * 32 + (__ffs(who) - 1);     // lowest lane = lowest id
+      }
     }
-    if (lane == 0) st.choice[r] = (bi == 0x7fffffff) ? 0 : bi;
+  }
+  __syncthreads();
+  for (int r = threadIdx.x; r < B; r += 128) {
+    if (!st.active[r]) continue;
+    uint32_t bk = s_key[0][r];
+    int bi = s_id[0][r];
+#pragma unroll
+    for (int w = 1; w < 4; ++w)
+      if (s_key[w][r] > bk) { bk = s_key[w][r]; bi = s_id[w][r]; }     // warps ascend in id: '>' keeps the lowest
+    tile_val[(size_t)r * n_tiles + tile] = __uint_as_float(bk);       // order key, bit-cast
+    tile_idx[(size_t)r * n_tiles + tile] = bi;
   }
 }
 
 // ------------------------------------------------------------------------------------ step bookkeeping
-// One block, one thread per row.  is_prefill: the prompt has just been cached (ctx_len set by the
-// host) and this is generated token 1; otherwise the fed token becomes part of the cache.
-__global__ void __launch_bounds__(kMaxBatch)
-bookkeeping_kernel(RowState st, const int32_t* __restrict__ forced, int32_t* __restrict__ next_tokens, int B,
-                   int eos_id, int is_prefill) {
+// One block of 1024 threads; warp w serves rows w, w+32, ...: final argmax over the vocabulary
+// tiles, then the row's state update.  is_prefill: the prompt has just been cached (ctx_len set
+// by the host) and this is generated token 1; otherwise the fed token becomes part of the cache.
+__global__ void __launch_bounds__(1024)
+bookkeeping_kernel(RowState st, const float* __restrict__ tile_val, const int32_t* __restrict__ tile_idx, int n_tiles,
+                   const int32_t* __restrict__ forced, int32_t* __restrict__ next_tokens, int B, int eos_id,
+                   int is_prefill) {
+  __shared__ int s_still;
   pdl_launch_dependents();
   pdl_wait();
-  const int r = threadIdx.x;
+  if (threadIdx.x == 0) s_still = 0;
+  __syncthreads();
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   int still = 0;
-  if (r < B) {
+  for (int r = warp; r < B; r += 32) {
     int tok = eos_id;
     if (st.active[r]) {
-      if (!is_prefill) st.ctx_len[r] += 1;
-      const int cap = st.scalars[0];
-      const int gidx = st.gen[r] + 1;                 // 1-based index of the token being emitted
-      tok = st.choice[r];
-      if (st.eos_at[r] > 0 && gidx == st.eos_at[r]) tok = eos_id;
-      if (forced) tok = forced[r];
-      st.out_tokens[(size_t)r * st.max_new + (gidx - 1)] = tok;
-      st.gen[r] = gidx;
-      st.cur_tok[r] = tok;
-      if (tok == eos_id) { st.finished[r] = 1; st.active[r] = 0; }
-      else if (gidx >= cap) { st.active[r] = 0; }
-      else still = 1;
+      uint32_t bk = 0;
+      int bi = 0x7fffffff;
+      for (int t = lane; t < n_tiles; t += 32) {
+        const uint32_t k = __float_as_uint(tile_val[(size_t)r * n_tiles + t]);
+        const int id = tile_idx[(size_t)r * n_tiles + t];
+        if (k > bk || (k == bk && id < bi)) { bk = k; bi = id; }
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const uint32_t ok = __shfl_xor_sync(0xffffffffu, bk, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (ok > bk || (ok == bk && oi < bi)) { bk = ok; bi = oi; }
+      }
+      if (lane == 0) {
+        if (!is_prefill) st.ctx_len[r] += 1;
+        const int cap = st.scalars[0];
+        const int gidx = st.gen[r] + 1;               // 1-based index of the token being emitted
+        tok = (bi == 0x7fffffff) ? 0 : bi;
+        if (st.eos_at[r] > 0 && gidx == st.eos_at[r]) tok = eos_id;
+        if (forced) tok = forced[r];
+        st.out_tokens[(size_t)r * st.max_new + (gidx - 1)] = tok;
+        st.gen[r] = gidx;
+        st.cur_tok[r] = tok;
+        if (tok == eos_id) { st.finished[r] = 1; st.active[r] = 0; }
+        else if (gidx >= cap) { st.active[r] = 0; }
+        else still += 1;
+      }
     }
-    if (next_tokens) next_tokens[r] = tok;
+    if (lane == 0 && next_tokens) next_tokens[r] = tok;
   }
-  const int c = __syncthreads_count(still);
-  if (threadIdx.x == 0) st.scalars[1] = c;
+  if (lane == 0 && still) atomicAdd(&s_still, still);
+  __syncthreads();
+  if (threadIdx.x == 0) st.scalars[1] = s_still;
 }
 
 // ------------------------------------------------------------------------------------ prompt-pass kernels

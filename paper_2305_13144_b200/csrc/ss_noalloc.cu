@@ -71,7 +71,7 @@ noalloc_rmsnorm_kernel(const float* __restrict__ h, const __nv_bfloat16* __restr
 __global__ void __launch_bounds__(256)
 noalloc_reduce_kernel(const float* __restrict__ partial, SplitInfo sp, float* __restrict__ logits, int V) {
   const int r = blockIdx.y, v = blockIdx.x * blockDim.x + threadIdx.x;
-  if (v < V) logits[(size_t)r * V + v] = sum_partials(partial, sp, v, r);
+  if (v < V) logits[(size_t)r * V + v] = sum_partials_derived(partial, sp, v, r);
 }
 
 int setup_device(int dev, DeviceSetup** out) {
@@ -165,7 +165,7 @@ extern "C" int ss_logits_noalloc(const float* hidden, const void* norm_gain, con
   a.status = status;
   gemm_wx_kernel<<<dim3(1, p.gridx), kGemmThreads, p.smem_bytes, st>>>(mw, mx, a);
   SplitInfo sp;
-  sp.gridx = p.gridx; sp.kb = p.kb; sp.max_seg = p.max_seg; sp.NT = p.NT; sp.total = total;
+  sp.gridx = p.gridx; sp.kb = p.kb; sp.max_seg = p.max_seg; sp.NT = p.NT; sp.total = total; sp.tiles = nullptr;
   noalloc_reduce_kernel<<<dim3((vocab + 255) / 256, n_rows), 256, 0, st>>>(partial, sp, logits, vocab);
   return cudaGetLastError() == cudaSuccess ? SS_OK : SS_ERR_CUDA;
 }

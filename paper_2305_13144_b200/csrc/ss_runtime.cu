@@ -57,14 +57,28 @@ GemmPlan plan_gemm(int n_out, int K, int NT, int tok_tiles, int mode, int n_sm) 
   return p;
 }
 
-SplitInfo split_of(const GemmPlan& p) {
+SplitInfo split_of(const GemmPlan& p, const TileSeg* tiles) {
   SplitInfo s;
   s.gridx = p.gridx;
   s.kb = p.kb;
   s.max_seg = p.max_seg;
   s.NT = p.NT;
   s.total = (long long)p.n_tiles * p.kb;
+  s.tiles = tiles;
   return s;
+}
+
+// Per tile: where its partial segments live (depends on the split only, not on the token tile).
+std::vector<TileSeg> tile_table(const GemmPlan& p) {
+  SplitInfo s = split_of(p, nullptr);
+  std::vector<TileSeg> t(p.n_tiles);
+  for (int tile = 0; tile < p.n_tiles; ++tile) {
+    const long long x0 = (long long)tile * p.kb;
+    const int c0 = split_owner(s, x0), c1 = split_owner(s, x0 + p.kb - 1);
+    const int seg0 = tile - (int)(split_begin(s, c0) / p.kb);
+    t[tile] = {c0 * p.max_seg + seg0, c0 + 1, c1, 0};
+  }
+  return t;
 }
 
 }  // namespace
@@ -107,6 +121,10 @@ struct ss_ctx {
   size_t partial_bytes = 0;
   float *part_ml = nullptr, *part_acc = nullptr;
   int max_chunks = 0;
+  TileSeg* tbl[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};   // qkv, o, gate/up, down, lm head
+  float* tile_val = nullptr;       // [kMaxBatch][n_tiles of the vocabulary]
+  int32_t* tile_idx = nullptr;
+  int n_tiles_lm = 0;
   // tensor maps for activation operands, keyed by (buffer id, box rows)
   std::map<std::pair<int, int>, CUtensorMap> xmaps;
 
@@ -225,6 +243,7 @@ struct Offsets {
   std::vector<size_t> attn_norm, wqkv, wo, ffn_norm, wgu, wdown;
   size_t inv_freq, status, rows, block_table, out_tokens, tok, h, x, qkv, attn_o, gu, act;
   size_t h_dec, x_dec, q_dec, o_dec, act_dec, partial, part_ml, part_acc, kv;
+  size_t tbl[5], tile_val, tile_idx;
   size_t partial_bytes;
   int R, max_pages, n_pages, max_chunks;
   size_t total;
@@ -290,6 +309,9 @@ void layout(const ss_model_cfg& m, const ss_runtime_cfg& rt, int n_sm, Offsets& 
   o.max_chunks = ceil_div(rt.max_ctx, kAttnChunk);
   o.part_ml = a.take((size_t)kMaxBatch * m.n_heads * o.max_chunks * 2 * 4);
   o.part_acc = a.take((size_t)kMaxBatch * m.n_heads * o.max_chunks * m.head_dim * 4);
+  for (int i = 0; i < 5; ++i) o.tbl[i] = a.take((size_t)ceil_div(shapes[i][0], kTileM) * sizeof(TileSeg));
+  o.tile_val = a.take((size_t)kMaxBatch * ceil_div((int)V, kTileM) * 4);
+  o.tile_idx = a.take((size_t)kMaxBatch * ceil_div((int)V, kTileM) * 4);
   o.n_pages = (int)((rt.kv_pool_tokens + kPageTokens - 1) / kPageTokens) + rt.max_batch;
   const size_t page_bytes = (size_t)2 * m.n_heads * kPageTokens * m.head_dim * 2;
   o.kv = a.take((size_t)std::max(1, m.n_layers) * o.n_pages * page_bytes);
@@ -361,8 +383,8 @@ int enqueue_decode_step(ss_ctx* c, const ss_step_opts* opts, int32_t* next_token
   for (int l = 0; l < m.n_layers; ++l) {
     const LayerWeights& w = c->layers[l];
     if ((rc = run_gemm(c, w.m_qkv, *mx, p_qkv, kGemmPartial, B, nullptr, nullptr, 0))) return rc;
-    SS_CUDA(c, launch(c, rope_append_decode_kernel, dim3(H, B), dim3(Dh / 2), 0, (const float*)c->partial,
-                      split_of(p_qkv), c->st, c->kv, l, (const float*)c->inv_freq, c->q_dec, d, c->status));
+    SS_CUDA(c, launch(c, rope_append_decode_kernel, dim3(H, B), dim3(Dh), 0, (const float*)c->partial,
+                      split_of(p_qkv, c->tbl[0]), c->st, c->kv, l, (const float*)c->inv_freq, c->q_dec, d, c->status));
     aa.layer = l;
     if (Dh == 128) {
       SS_CUDA(c, launch(c, attn_decode_kernel<128>, dim3(attn_grid), dim3(128), 0, aa));
@@ -372,26 +394,28 @@ int enqueue_decode_step(ss_ctx* c, const ss_step_opts* opts, int32_t* next_token
       SS_CUDA(c, launch(c, attn_combine_kernel<64>, dim3(H, B), dim3(64), 0, aa));
     }
     if ((rc = run_gemm(c, w.m_o, *mo, p_o, kGemmPartial, B, nullptr, nullptr, 0))) return rc;
-    SS_CUDA(c, launch(c, residual_rmsnorm_partial_kernel, dim3(B), dim3(256), 0, (const float*)c->partial,
-                      split_of(p_o), (const int32_t*)c->st.active, c->h_dec, (const bf16*)w.ffn_norm, c->x_dec,
+    SS_CUDA(c, launch(c, residual_rmsnorm_partial_kernel, dim3(B), dim3(1024), 0, (const float*)c->partial,
+                      split_of(p_o, c->tbl[1]), (const int32_t*)c->st.active, c->h_dec, (const bf16*)w.ffn_norm, c->x_dec,
                       (float*)nullptr, d, m.rms_eps));
     if ((rc = run_gemm(c, w.m_gu, *mx, p_gu, kGemmPartial, B, nullptr, nullptr, 0))) return rc;
     SS_CUDA(c, launch(c, swiglu_partial_kernel, dim3(ceil_div(F, 256), B), dim3(256), 0, (const float*)c->partial,
-                      split_of(p_gu), c->act_dec, F));
+                      split_of(p_gu, c->tbl[2]), c->act_dec, F));
     if ((rc = run_gemm(c, w.m_down, *ma, p_dn, kGemmPartial, B, nullptr, nullptr, 0))) return rc;
     const bool last = l + 1 == m.n_layers;
     const bf16* next_norm = last ? c->final_norm : c->layers[l + 1].attn_norm;
-    SS_CUDA(c, launch(c, residual_rmsnorm_partial_kernel, dim3(B), dim3(256), 0, (const float*)c->partial,
-                      split_of(p_dn), (const int32_t*)c->st.active, c->h_dec, next_norm, c->x_dec,
+    SS_CUDA(c, launch(c, residual_rmsnorm_partial_kernel, dim3(B), dim3(1024), 0, (const float*)c->partial,
+                      split_of(p_dn, c->tbl[3]), (const int32_t*)c->st.active, c->h_dec, next_norm, c->x_dec,
                       (last && opts) ? opts->dump_hidden : (float*)nullptr, d, m.rms_eps));
   }
   if (m.n_layers == 0 && opts && opts->dump_hidden)
     SS_CUDA(c, cudaMemcpyAsync(opts->dump_hidden, c->h_dec, (size_t)B * d * 4, cudaMemcpyDeviceToDevice, c->stream));
   if ((rc = run_gemm(c, c->m_lm, *mx, p_lm, kGemmPartial, B, nullptr, nullptr, 0))) return rc;
-  SS_CUDA(c, launch(c, lmhead_argmax_kernel, dim3(B), dim3(1024), 0, (const float*)c->partial, split_of(p_lm), c->st,
-                    opts ? opts->dump_logits : (float*)nullptr, V, m.eos_id));
-  SS_CUDA(c, launch(c, bookkeeping_kernel, dim3(1), dim3(kMaxBatch), 0, c->st,
-                    opts ? opts->forced_tokens : (const int32_t*)nullptr, next_tokens, B, m.eos_id, 0));
+  SS_CUDA(c, launch(c, lmhead_tile_argmax_kernel, dim3(c->n_tiles_lm), dim3(128), 0, (const float*)c->partial,
+                    split_of(p_lm, c->tbl[4]), c->st, opts ? opts->dump_logits : (float*)nullptr, c->tile_val,
+                    c->tile_idx, B, V, c->n_tiles_lm, m.eos_id));
+  SS_CUDA(c, launch(c, bookkeeping_kernel, dim3(1), dim3(1024), 0, c->st, (const float*)c->tile_val,
+                    (const int32_t*)c->tile_idx, c->n_tiles_lm, opts ? opts->forced_tokens : (const int32_t*)nullptr,
+                    next_tokens, B, m.eos_id, 0));
   return SS_OK;
 }
 
@@ -551,6 +575,18 @@ int ss_create(const ss_model_cfg* model, const ss_runtime_cfg* rt, void* dev_are
   c->part_ml = (float*)(A + o.part_ml);
   c->part_acc = (float*)(A + o.part_acc);
   c->max_chunks = o.max_chunks;
+  c->tile_val = (float*)(A + o.tile_val);
+  c->tile_idx = (int32_t*)(A + o.tile_idx);
+  c->n_tiles_lm = ceil_div((int)V, kTileM);
+  {
+    const int shp[5][2] = {{(int)(3 * d), (int)d}, {(int)d, (int)d}, {(int)(2 * F), (int)d}, {(int)d, (int)F}, {(int)V, (int)d}};
+    for (int i = 0; i < 5; ++i) {
+      c->tbl[i] = (TileSeg*)(A + o.tbl[i]);
+      const std::vector<TileSeg> t = tile_table(plan_gemm(shp[i][0], shp[i][1], 16, 1, kGemmPartial, c->n_sm));
+      if (cudaMemcpy(c->tbl[i], t.data(), t.size() * sizeof(TileSeg), cudaMemcpyHostToDevice) != cudaSuccess)
+        return fail(SS_ERR_CUDA);
+    }
+  }
   c->kv.pool = (bf16*)(A + o.kv);
   c->kv.page_elems = (size_t)2 * model->n_heads * kPageTokens * model->head_dim;
   c->kv.layer_stride = (size_t)o.n_pages * c->kv.page_elems;
@@ -710,10 +746,12 @@ int ss_prefill(ss_ctx* c, const int32_t* tokens, const int32_t* cu, int32_t B, c
   if ((rc = xmap(c, 3, NT, &mx))) return bail(rc);
   const GemmPlan p_lm = plan_gemm(m.vocab, m.d_model, NT, 1, kGemmPartial, c->n_sm);
   if ((rc = run_gemm(c, c->m_lm, *mx, p_lm, kGemmPartial, B, nullptr, nullptr, 0))) return bail(rc);
-  SS_CUDA_B(launch(c, lmhead_argmax_kernel, dim3(B), dim3(1024), 0, (const float*)c->partial, split_of(p_lm), c->st,
-                   opts ? opts->dump_logits : (float*)nullptr, m.vocab, m.eos_id));
-  SS_CUDA_B(launch(c, bookkeeping_kernel, dim3(1), dim3(kMaxBatch), 0, c->st,
-                   opts ? opts->forced_tokens : (const int32_t*)nullptr, first_tokens, B, m.eos_id, 1));
+  SS_CUDA_B(launch(c, lmhead_tile_argmax_kernel, dim3(c->n_tiles_lm), dim3(128), 0, (const float*)c->partial,
+                   split_of(p_lm, c->tbl[4]), c->st, opts ? opts->dump_logits : (float*)nullptr, c->tile_val,
+                   c->tile_idx, B, m.vocab, c->n_tiles_lm, m.eos_id));
+  SS_CUDA_B(launch(c, bookkeeping_kernel, dim3(1), dim3(1024), 0, c->st, (const float*)c->tile_val,
+                   (const int32_t*)c->tile_idx, c->n_tiles_lm, opts ? opts->forced_tokens : (const int32_t*)nullptr,
+                   first_tokens, B, m.eos_id, 1));
 #undef SS_CUDA_B
   return SS_OK;
 }
