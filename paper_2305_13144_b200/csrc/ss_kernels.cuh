@@ -60,6 +60,26 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
   return t;
 }
 
+// ------------------------------------------------------------------------------------ weight repacking
+// Row-major [rows, K] bf16 -> the GEMM's streaming layout: 16 KiB blocks in (tile, k-block) order, each
+// the exact shared-memory image of a 128-row x 64-column tile under the 128-byte swizzle (row r at
+// r*128 bytes, its 16-byte chunk c stored at chunk position c ^ (r & 7)).  One thread per 16-byte chunk.
+// row_off places the source at a row offset of the destination matrix (q,k,v and gate,up are stacked).
+__global__ void __launch_bounds__(256)
+repack_weights_kernel(const uint4* __restrict__ src, long long rows, int K, uint8_t* __restrict__ dst, int row_off,
+                      int kb) {
+  const int chunks_per_row = K >> 3;
+  const long long id = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (id >= rows * chunks_per_row) return;
+  const long long sr = id / chunks_per_row;
+  const int cc = (int)(id - sr * chunks_per_row);
+  const long long n = row_off + sr;
+  const long long tile = n >> 7;
+  const int r = (int)(n & 127), k = cc >> 3, c = cc & 7;
+  uint8_t* blk = dst + ((size_t)tile * kb + k) * (size_t)(kTileM * kTileK * 2);
+  *reinterpret_cast<uint4*>(blk + r * 128 + ((c ^ (r & 7)) << 4)) = src[id];
+}
+
 // ------------------------------------------------------------------------------------ embedding + first norm
 // h[row] = E[token]; x[row] = RMSNorm(h[row]) * g   (rows: decode B rows or T prompt tokens)
 __global__ void __launch_bounds__(256)
