@@ -75,6 +75,14 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       : "r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y), "l"(hint)
       : "memory");
 }
+// Linear bulk copy global -> shared (both 16-byte aligned, size a multiple of 16).
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t hint) {
+  asm volatile(
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+      :
+      : "r"(dst), "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(bar), "l"(hint)
+      : "memory");
+}
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");
 }
@@ -211,7 +219,7 @@ gemm_wx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
       mbar_init(smem_u32(&hdr->acc_empty[b]), 4);
     }
     fence_barrier_init();
-    tma_prefetch_desc(&map_w);
+    if (!a.w_tiled) tma_prefetch_desc(&map_w);
     tma_prefetch_desc(&map_x);
   }
   if (warp == 1) {
@@ -231,13 +239,17 @@ gemm_wx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(hint_w));
       asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(hint_x));
       const int pre = n_it < p.stages ? n_it : p.stages;
+      // Repacked weights: iteration `it` of the (tile, k-block) space is the 16 KiB block number `it`,
+      // already in the swizzled shared-memory image, so a CTA's whole range is one contiguous span.
+      const uint8_t* w_tiled = reinterpret_cast<const uint8_t*>(a.w_tiled);
       // phase 1: weight tiles of the first ring fill, before the dependency resolves
       for (int i = 0; i < pre; ++i) {
         const long long it = it0 + i;
         const int tile = (int)(it / p.kb), kblk = (int)(it % p.kb);
         const uint32_t full = smem_u32(&hdr->full[i]);
         mbar_expect_tx(full, stage_bytes);
-        tma_load_2d(stage0 + i * stage_bytes, &map_w, full, kblk * kTileK, tile * kTileM, hint_w);
+        if (w_tiled) bulk_load(stage0 + i * stage_bytes, w_tiled + (size_t)it * a_bytes, a_bytes, full, hint_w);
+        else tma_load_2d(stage0 + i * stage_bytes, &map_w, full, kblk * kTileK, tile * kTileM, hint_w);
       }
       pdl_wait();
       for (int i = 0; i < pre; ++i) {
@@ -255,7 +267,8 @@ gemm_wx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         if (!mbar_wait(smem_u32(&hdr->empty[stage]), phase ^ 1u, a.status, kStatusProducerTimeout)) break;
         const uint32_t full = smem_u32(&hdr->full[stage]);
         mbar_expect_tx(full, stage_bytes);
-        tma_load_2d(stage0 + stage * stage_bytes, &map_w, full, kblk * kTileK, tile * kTileM, hint_w);
+        if (w_tiled) bulk_load(stage0 + stage * stage_bytes, w_tiled + (size_t)it * a_bytes, a_bytes, full, hint_w);
+        else tma_load_2d(stage0 + stage * stage_bytes, &map_w, full, kblk * kTileK, tile * kTileM, hint_w);
         tma_load_2d(stage0 + stage * stage_bytes + a_bytes, &map_x, full, kblk * kTileK, tok_tile * p.NT, hint_x);
         if (++stage == p.stages) { stage = 0; phase ^= 1u; }
       }

@@ -52,6 +52,7 @@ struct GemmPlan {
 
 struct GemmArgs {
   GemmPlan p;
+  const void* w_tiled; // weights repacked as contiguous 16 KiB (tile, k-block) images, or null (row-major via TMA)
   int mode;
   int n_tok;           // valid tokens
   float* partial;      // [gridx*max_seg][NT][128]

@@ -25,10 +25,15 @@ inline size_t align_up(size_t x, size_t a = kAlign) { return (x + a - 1) / a * a
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 inline int round_up(int a, int b) { return ceil_div(a, b) * b; }
 
+// Projection matrices live in the tiled streaming layout (see repack_weights_kernel).
 struct LayerWeights {
-  bf16 *attn_norm, *wqkv, *wo, *ffn_norm, *wgu, *wdown;
-  CUtensorMap m_qkv, m_o, m_gu, m_down;
+  bf16 *attn_norm, *ffn_norm;
+  uint8_t *wqkv, *wo, *wgu, *wdown;
 };
+
+inline size_t tiled_bytes(int64_t n_out, int64_t K) {
+  return (size_t)ceil_div((int)n_out, kTileM) * ceil_div((int)K, kTileK) * (size_t)(kTileM * kTileK * 2);
+}
 
 GemmPlan plan_gemm(int n_out, int K, int NT, int tok_tiles, int mode, int n_sm) {
   GemmPlan p{};
@@ -99,9 +104,11 @@ struct ss_ctx {
   uint8_t* arena = nullptr;
   size_t arena_bytes = 0;
   // weights
-  bf16 *embed = nullptr, *lm_head = nullptr, *final_norm = nullptr;
+  bf16 *embed = nullptr, *final_norm = nullptr;
+  uint8_t* lm_head = nullptr;
+  uint8_t* staging = nullptr;      // one row-major tensor on its way into the tiled layout
+  size_t staging_bytes = 0;
   std::vector<LayerWeights> layers;
-  CUtensorMap m_lm;
   std::vector<uint8_t> loaded;     // per tensor slot
   int n_loaded = 0, n_expected = 0;
   // misc device
@@ -210,10 +217,11 @@ int xmap(ss_ctx* c, int id, int box_rows, const CUtensorMap** out) {
   return SS_OK;
 }
 
-int run_gemm(ss_ctx* c, const CUtensorMap& mw, const CUtensorMap& mx, const GemmPlan& p, int mode, int n_tok,
+int run_gemm(ss_ctx* c, const uint8_t* w_tiled, const CUtensorMap& mx, const GemmPlan& p, int mode, int n_tok,
              void* out_bf16, float* out_f32, int ld_out) {
   GemmArgs a{};
   a.p = p;
+  a.w_tiled = w_tiled;
   a.mode = mode;
   a.n_tok = n_tok;
   a.partial = c->partial;
@@ -225,7 +233,8 @@ int run_gemm(ss_ctx* c, const CUtensorMap& mw, const CUtensorMap& mx, const Gemm
     const size_t need = (size_t)p.gridx * p.max_seg * p.NT * 128 * sizeof(float);
     if (need > c->partial_bytes) return SS_ERR_CAPACITY;
   }
-  SS_CUDA(c, launch(c, gemm_wx_kernel, dim3(p.gridy, p.gridx), dim3(kGemmThreads), (size_t)p.smem_bytes, mw, mx, a));
+  // the weight tensor map is unused with tiled weights; the activation map stands in for it
+  SS_CUDA(c, launch(c, gemm_wx_kernel, dim3(p.gridy, p.gridx), dim3(kGemmThreads), (size_t)p.smem_bytes, mx, mx, a));
   return SS_OK;
 }
 
@@ -239,7 +248,7 @@ struct ArenaPlan {
 };
 
 struct Offsets {
-  size_t embed, lm_head, final_norm;
+  size_t embed, lm_head, final_norm, staging, staging_bytes, weights_end;
   std::vector<size_t> attn_norm, wqkv, wo, ffn_norm, wgu, wdown;
   size_t inv_freq, status, rows, block_table, out_tokens, tok, h, x, qkv, attn_o, gu, act;
   size_t h_dec, x_dec, q_dec, o_dec, act_dec, partial, part_ml, part_acc, kv;
@@ -269,14 +278,17 @@ void layout(const ss_model_cfg& m, const ss_runtime_cfg& rt, int n_sm, Offsets& 
   o.ffn_norm.resize(m.n_layers); o.wgu.resize(m.n_layers); o.wdown.resize(m.n_layers);
   for (int l = 0; l < m.n_layers; ++l) {
     o.attn_norm[l] = a.take(d * 2);
-    o.wqkv[l] = a.take(3 * d * d * 2);
-    o.wo[l] = a.take(d * d * 2);
+    o.wqkv[l] = a.take(tiled_bytes(3 * d, d));
+    o.wo[l] = a.take(tiled_bytes(d, d));
     o.ffn_norm[l] = a.take(d * 2);
-    o.wgu[l] = a.take(2 * F * d * 2);
-    o.wdown[l] = a.take(d * F * 2);
+    o.wgu[l] = a.take(tiled_bytes(2 * F, d));
+    o.wdown[l] = a.take(tiled_bytes(d, F));
   }
   o.final_norm = a.take(d * 2);
-  o.lm_head = a.take(V * d * 2);
+  o.lm_head = a.take(tiled_bytes(V, d));
+  o.weights_end = a.total;
+  o.staging_bytes = std::max(std::max(V * d, F * d), d * d) * 2;
+  o.staging = a.take(o.staging_bytes);
   o.inv_freq = a.take(m.head_dim / 2 * sizeof(float));
   o.status = a.take(64);
   o.rows = a.take((size_t)kMaxBatch * 4 * 8 + 64);           // 7 row arrays + scalars
@@ -327,12 +339,21 @@ int query_sms() {
   return n;
 }
 
-int weight_slot(const ss_ctx* c, const std::string& name, bf16** dst, int64_t* rows, int64_t* cols, int* slot) {
+struct WeightSlot {
+  void* dst;          // plain tensors: destination; tiled: base of the tiled matrix
+  int64_t rows, cols; // expected shape of the source
+  int slot;
+  bool tiled;
+  int row_off;        // tiled: row offset inside the stacked matrix
+};
+
+int weight_slot(const ss_ctx* c, const std::string& name, WeightSlot* out) {
   const int64_t d = c->m.d_model, F = c->m.d_ffn, V = c->m.vocab;
-  auto set = [&](bf16* p, int64_t r, int64_t cc, int s) { *dst = p; *rows = r; *cols = cc; *slot = s; return SS_OK; };
-  if (name == "embed") return set(c->embed, V, d, 0);
-  if (name == "lm_head") return set(c->lm_head, V, d, 1);
-  if (name == "final_norm") return set(c->final_norm, 1, d, 2);
+  auto plain = [&](void* p, int64_t r, int64_t cc, int s) { *out = {p, r, cc, s, false, 0}; return SS_OK; };
+  auto tiled = [&](void* p, int64_t r, int64_t cc, int s, int64_t off) { *out = {p, r, cc, s, true, (int)off}; return SS_OK; };
+  if (name == "embed") return plain(c->embed, V, d, 0);
+  if (name == "lm_head") return tiled(c->lm_head, V, d, 1, 0);
+  if (name == "final_norm") return plain(c->final_norm, 1, d, 2);
   if (name.size() > 2 && name[0] == 'l') {
     size_t dot = name.find('.');
     if (dot == std::string::npos) return SS_ERR_ARG;
@@ -341,15 +362,15 @@ int weight_slot(const ss_ctx* c, const std::string& name, bf16** dst, int64_t* r
     const std::string k = name.substr(dot + 1);
     const LayerWeights& w = c->layers[l];
     const int base = 3 + l * 9;
-    if (k == "attn_norm") return set(w.attn_norm, 1, d, base + 0);
-    if (k == "wq") return set(w.wqkv, d, d, base + 1);
-    if (k == "wk") return set(w.wqkv + d * d, d, d, base + 2);
-    if (k == "wv") return set(w.wqkv + 2 * d * d, d, d, base + 3);
-    if (k == "wo") return set(w.wo, d, d, base + 4);
-    if (k == "ffn_norm") return set(w.ffn_norm, 1, d, base + 5);
-    if (k == "w_gate") return set(w.wgu, F, d, base + 6);
-    if (k == "w_up") return set(w.wgu + F * d, F, d, base + 7);
-    if (k == "w_down") return set(w.wdown, d, F, base + 8);
+    if (k == "attn_norm") return plain(w.attn_norm, 1, d, base + 0);
+    if (k == "wq") return tiled(w.wqkv, d, d, base + 1, 0);
+    if (k == "wk") return tiled(w.wqkv, d, d, base + 2, d);
+    if (k == "wv") return tiled(w.wqkv, d, d, base + 3, 2 * d);
+    if (k == "wo") return tiled(w.wo, d, d, base + 4, 0);
+    if (k == "ffn_norm") return plain(w.ffn_norm, 1, d, base + 5);
+    if (k == "w_gate") return tiled(w.wgu, F, d, base + 6, 0);
+    if (k == "w_up") return tiled(w.wgu, F, d, base + 7, F);
+    if (k == "w_down") return tiled(w.wdown, d, F, base + 8, 0);
   }
   return SS_ERR_ARG;
 }
@@ -382,7 +403,7 @@ int enqueue_decode_step(ss_ctx* c, const ss_step_opts* opts, int32_t* next_token
   const int attn_grid = c->n_sm * 4;
   for (int l = 0; l < m.n_layers; ++l) {
     const LayerWeights& w = c->layers[l];
-    if ((rc = run_gemm(c, w.m_qkv, *mx, p_qkv, kGemmPartial, B, nullptr, nullptr, 0))) return rc;
+    if ((rc = run_gemm(c, w.wqkv, *mx, p_qkv, kGemmPartial, B, nullptr, nullptr, 0))) return rc;
     SS_CUDA(c, launch(c, rope_append_decode_kernel, dim3(H, B), dim3(Dh), 0, (const float*)c->partial,
                       split_of(p_qkv, c->tbl[0]), c->st, c->kv, l, (const float*)c->inv_freq, c->q_dec, d, c->status));
     aa.layer = l;
@@ -393,14 +414,14 @@ int enqueue_decode_step(ss_ctx* c, const ss_step_opts* opts, int32_t* next_token
       SS_CUDA(c, launch(c, attn_decode_kernel<64>, dim3(attn_grid), dim3(128), 0, aa));
       SS_CUDA(c, launch(c, attn_combine_kernel<64>, dim3(H, B), dim3(64), 0, aa));
     }
-    if ((rc = run_gemm(c, w.m_o, *mo, p_o, kGemmPartial, B, nullptr, nullptr, 0))) return rc;
+    if ((rc = run_gemm(c, w.wo, *mo, p_o, kGemmPartial, B, nullptr, nullptr, 0))) return rc;
     SS_CUDA(c, launch(c, residual_rmsnorm_partial_kernel, dim3(B), dim3(1024), 0, (const float*)c->partial,
                       split_of(p_o, c->tbl[1]), (const int32_t*)c->st.active, c->h_dec, (const bf16*)w.ffn_norm, c->x_dec,
                       (float*)nullptr, d, m.rms_eps));
-    if ((rc = run_gemm(c, w.m_gu, *mx, p_gu, kGemmPartial, B, nullptr, nullptr, 0))) return rc;
+    if ((rc = run_gemm(c, w.wgu, *mx, p_gu, kGemmPartial, B, nullptr, nullptr, 0))) return rc;
     SS_CUDA(c, launch(c, swiglu_partial_kernel, dim3(ceil_div(F, 256), B), dim3(256), 0, (const float*)c->partial,
                       split_of(p_gu, c->tbl[2]), c->act_dec, F));
-    if ((rc = run_gemm(c, w.m_down, *ma, p_dn, kGemmPartial, B, nullptr, nullptr, 0))) return rc;
+    if ((rc = run_gemm(c, w.wdown, *ma, p_dn, kGemmPartial, B, nullptr, nullptr, 0))) return rc;
     const bool last = l + 1 == m.n_layers;
     const bf16* next_norm = last ? c->final_norm : c->layers[l + 1].attn_norm;
     SS_CUDA(c, launch(c, residual_rmsnorm_partial_kernel, dim3(B), dim3(1024), 0, (const float*)c->partial,
@@ -409,7 +430,7 @@ int enqueue_decode_step(ss_ctx* c, const ss_step_opts* opts, int32_t* next_token
   }
   if (m.n_layers == 0 && opts && opts->dump_hidden)
     SS_CUDA(c, cudaMemcpyAsync(opts->dump_hidden, c->h_dec, (size_t)B * d * 4, cudaMemcpyDeviceToDevice, c->stream));
-  if ((rc = run_gemm(c, c->m_lm, *mx, p_lm, kGemmPartial, B, nullptr, nullptr, 0))) return rc;
+  if ((rc = run_gemm(c, c->lm_head, *mx, p_lm, kGemmPartial, B, nullptr, nullptr, 0))) return rc;
   SS_CUDA(c, launch(c, lmhead_tile_argmax_kernel, dim3(c->n_tiles_lm), dim3(128), 0, (const float*)c->partial,
                     split_of(p_lm, c->tbl[4]), c->st, opts ? opts->dump_logits : (float*)nullptr, c->tile_val,
                     c->tile_idx, B, V, c->n_tiles_lm, m.eos_id));
@@ -440,7 +461,7 @@ int enqueue_prefill_chunk(ss_ctx* c, int s0, int s1, const int32_t* cu, int T) {
                     (const bf16*)c->embed, first_norm, c->h, c->x, d, m.rms_eps, V));
   for (int l = 0; l < m.n_layers; ++l) {
     const LayerWeights& w = c->layers[l];
-    if ((rc = run_gemm(c, w.m_qkv, *mx, p_qkv, kGemmDirectBf16, T, c->qkv, nullptr, 3 * d))) return rc;
+    if ((rc = run_gemm(c, w.wqkv, *mx, p_qkv, kGemmDirectBf16, T, c->qkv, nullptr, 3 * d))) return rc;
     SS_CUDA(c, launch(c, rope_append_prefill_kernel, dim3(T, H), dim3(Dh / 2), 0, c->qkv, (const int32_t*)c->d_tok_row,
                       (const int32_t*)c->d_tok_pos, c->st, c->kv, l, (const float*)c->inv_freq, d, c->status));
     const dim3 ag(ceil_div(max_len, 32), H, nseq);
@@ -448,11 +469,11 @@ int enqueue_prefill_chunk(ss_ctx* c, int s0, int s1, const int32_t* cu, int T) {
       SS_CUDA(c, launch(c, attn_prefill_kernel<128>, ag, dim3(128), 0, (const bf16*)c->qkv, (const int32_t*)c->d_cu, c->attn_o, d));
     else
       SS_CUDA(c, launch(c, attn_prefill_kernel<64>, ag, dim3(128), 0, (const bf16*)c->qkv, (const int32_t*)c->d_cu, c->attn_o, d));
-    if ((rc = run_gemm(c, w.m_o, *mo, p_o, kGemmDirectF32Add, T, nullptr, c->h, d))) return rc;
+    if ((rc = run_gemm(c, w.wo, *mo, p_o, kGemmDirectF32Add, T, nullptr, c->h, d))) return rc;
     SS_CUDA(c, launch(c, rmsnorm_kernel, dim3(T), dim3(256), 0, (const float*)c->h, (const bf16*)w.ffn_norm, c->x, d, m.rms_eps));
-    if ((rc = run_gemm(c, w.m_gu, *mx, p_gu, kGemmDirectBf16, T, c->gu, nullptr, 2 * F))) return rc;
+    if ((rc = run_gemm(c, w.wgu, *mx, p_gu, kGemmDirectBf16, T, c->gu, nullptr, 2 * F))) return rc;
     SS_CUDA(c, launch(c, swiglu_kernel, dim3(T, ceil_div(F, 256)), dim3(256), 0, (const bf16*)c->gu, c->act, F));
-    if ((rc = run_gemm(c, w.m_down, *ma, p_dn, kGemmDirectF32Add, T, nullptr, c->h, d))) return rc;
+    if ((rc = run_gemm(c, w.wdown, *ma, p_dn, kGemmDirectF32Add, T, nullptr, c->h, d))) return rc;
     if (l + 1 < m.n_layers)
       SS_CUDA(c, launch(c, rmsnorm_kernel, dim3(T), dim3(256), 0, (const float*)c->h,
                         (const bf16*)c->layers[l + 1].attn_norm, c->x, d, m.rms_eps));
@@ -517,24 +538,23 @@ int ss_create(const ss_model_cfg* model, const ss_runtime_cfg* rt, void* dev_are
   c->arena_bytes = arena_bytes;
   const int64_t d = model->d_model, F = model->d_ffn, V = model->vocab;
   c->embed = (bf16*)(A + o.embed);
-  c->lm_head = (bf16*)(A + o.lm_head);
+  c->lm_head = A + o.lm_head;
+  c->staging = A + o.staging;
+  c->staging_bytes = o.staging_bytes;
   c->final_norm = (bf16*)(A + o.final_norm);
   c->layers.resize(model->n_layers);
   auto fail = [&](int code) { delete c; return code; };
   for (int l = 0; l < model->n_layers; ++l) {
     LayerWeights& w = c->layers[l];
     w.attn_norm = (bf16*)(A + o.attn_norm[l]);
-    w.wqkv = (bf16*)(A + o.wqkv[l]);
-    w.wo = (bf16*)(A + o.wo[l]);
+    w.wqkv = A + o.wqkv[l];
+    w.wo = A + o.wo[l];
     w.ffn_norm = (bf16*)(A + o.ffn_norm[l]);
-    w.wgu = (bf16*)(A + o.wgu[l]);
-    w.wdown = (bf16*)(A + o.wdown[l]);
-    if ((rc = make_map(c, &w.m_qkv, w.wqkv, 3 * d, d, kTileM))) return fail(rc);
-    if ((rc = make_map(c, &w.m_o, w.wo, d, d, kTileM))) return fail(rc);
-    if ((rc = make_map(c, &w.m_gu, w.wgu, 2 * F, d, kTileM))) return fail(rc);
-    if ((rc = make_map(c, &w.m_down, w.wdown, d, F, kTileM))) return fail(rc);
+    w.wgu = A + o.wgu[l];
+    w.wdown = A + o.wdown[l];
   }
-  if ((rc = make_map(c, &c->m_lm, c->lm_head, V, d, kTileM))) return fail(rc);
+  // tiles that reach beyond a matrix's rows or columns must read as zero
+  if (cudaMemsetAsync(A + o.embed, 0, o.weights_end - o.embed, c->stream) != cudaSuccess) return fail(SS_ERR_CUDA);
   c->n_expected = 3 + 9 * model->n_layers;
   c->loaded.assign(c->n_expected, 0);
   c->inv_freq = (float*)(A + o.inv_freq);
@@ -631,15 +651,32 @@ int ss_load_weights(ss_ctx* c, const ss_tensor_desc* t, int32_t n) {
   if (!c || (n > 0 && !t) || n < 0) return SS_ERR_ARG;
   for (int i = 0; i < n; ++i) {
     if (!t[i].name || !t[i].data) return SS_ERR_ARG;
-    bf16* dst;
-    int64_t rows, cols;
-    int slot;
-    int rc = weight_slot(c, t[i].name, &dst, &rows, &cols, &slot);
+    WeightSlot ws;
+    int rc = weight_slot(c, t[i].name, &ws);
     if (rc) return rc;
-    if (t[i].rows * t[i].cols != rows * cols || (rows > 1 && (t[i].rows != rows || t[i].cols != cols))) return SS_ERR_ARG;
-    SS_CUDA(c, cudaMemcpyAsync(dst, t[i].data, (size_t)rows * cols * 2,
-                               t[i].is_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, c->stream));
-    if (!c->loaded[slot]) { c->loaded[slot] = 1; c->n_loaded++; }
+    if (t[i].rows * t[i].cols != ws.rows * ws.cols || (ws.rows > 1 && (t[i].rows != ws.rows || t[i].cols != ws.cols)))
+      return SS_ERR_ARG;
+    const size_t bytes = (size_t)ws.rows * ws.cols * 2;
+    if (!ws.tiled) {
+      SS_CUDA(c, cudaMemcpyAsync(ws.dst, t[i].data, bytes,
+                                 t[i].is_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, c->stream));
+    } else {
+      const void* src = t[i].data;
+      if (!t[i].is_device || ((uintptr_t)src & 15)) {
+        if (bytes > c->staging_bytes) return SS_ERR_CAPACITY;
+        SS_CUDA(c, cudaMemcpyAsync(c->staging, src, bytes,
+                                   t[i].is_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, c->stream));
+        src = c->staging;
+      }
+      const long long chunks = (long long)ws.rows * (ws.cols / 8);
+      repack_weights_kernel<<<(unsigned)((chunks + 255) / 256), 256, 0, c->stream>>>(
+          (const uint4*)src, ws.rows, (int)ws.cols, (uint8_t*)ws.dst, ws.row_off, ceil_div((int)ws.cols, kTileK));
+      SS_CUDA(c, cudaGetLastError());
+      c->launches++;
+      // the staging buffer (or the caller's tensor) is free again once the repack has run
+      SS_CUDA(c, cudaStreamSynchronize(c->stream));
+    }
+    if (!c->loaded[ws.slot]) { c->loaded[ws.slot] = 1; c->n_loaded++; }
   }
   SS_CUDA(c, cudaStreamSynchronize(c->stream));
   return SS_OK;
@@ -745,7 +782,7 @@ int ss_prefill(ss_ctx* c, const int32_t* tokens, const int32_t* cu, int32_t B, c
   const CUtensorMap* mx;
   if ((rc = xmap(c, 3, NT, &mx))) return bail(rc);
   const GemmPlan p_lm = plan_gemm(m.vocab, m.d_model, NT, 1, kGemmPartial, c->n_sm);
-  if ((rc = run_gemm(c, c->m_lm, *mx, p_lm, kGemmPartial, B, nullptr, nullptr, 0))) return bail(rc);
+  if ((rc = run_gemm(c, c->lm_head, *mx, p_lm, kGemmPartial, B, nullptr, nullptr, 0))) return bail(rc);
   SS_CUDA_B(launch(c, lmhead_tile_argmax_kernel, dim3(c->n_tiles_lm), dim3(128), 0, (const float*)c->partial,
                    split_of(p_lm, c->tbl[4]), c->st, opts ? opts->dump_logits : (float*)nullptr, c->tile_val,
                    c->tile_idx, B, m.vocab, c->n_tiles_lm, m.eos_id));
