@@ -1,0 +1,798 @@
+// One decode step as ONE persistent cooperative kernel (one CTA per SM).
+//
+// Why: a decode step at small batch is a chain of ~130 weight-streaming projections separated by
+// tiny dependent stages.  As separate kernels every projection pays several microseconds of
+// launch, ramp-up and drain during which HBM idles.  Here a dedicated producer warp streams the
+// tiled weights of ALL projections of the step, in order, through one shared-memory ring; it
+// never waits for activations, so while the other warps sit in a grid barrier or run a small
+// stage, the ring keeps filling with the next projection's weights.
+//
+// Warp roles (352 threads):
+//   warp 0      weight producer: linear bulk copies of 16 KiB (tile, k-block) images into the ring
+//   warp 1      MMA issuer: tcgen05.mma, accumulators in tensor memory (two buffers)
+//   warp 2      activation loader: TMA loads of the [NT x 64] activation block of each ring stage,
+//               issued once the stage that produced the activations has passed its grid barrier
+//   warps 3-10  workers: drain accumulators to fp32 partials, then run the stage between two
+//               projections (partial sums in CTA order, RoPE, cache append, attention, residual,
+//               SwiGLU, arg-max, bookkeeping), separated by grid barriers
+//
+// RMSNorm is applied lazily: the residual stage writes x' = bf16(h * g) and per-slice sums of
+// squares; since a projection is linear, the consumer of its partial sums multiplies by
+// rsqrt(mean h^2 + eps).  This lets a row be split over many CTAs without a cross-CTA reduction.
+//
+// Every wait (mbarrier, grid barrier, flag) is bounded; on expiry the kernel records a status word,
+// raises a CTA-wide abort flag and all roles leave.
+#pragma once
+
+#include "ss_kernels.cuh"
+
+namespace ss {
+
+constexpr int kMegaThreads = 352;
+constexpr int kMegaWorkers = 256;          // warps 3..10
+constexpr int kMegaAttnChunk = 64;         // cached tokens per attention work item (one warp)
+constexpr int kRowSlice = 512;             // elements of a row handled by one residual work item
+constexpr int kMaxSlices = 16;             // d_model <= 8192
+
+enum : uint32_t { kStatusGridBarrierTimeout = 5, kStatusFlagTimeout = 6 };
+
+struct MegaGemmShape {
+  int n_tiles, kb, max_seg;
+  int gsplit;              // CTAs that share the iteration space (the others idle through this projection)
+  long long total;
+  const TileSeg* tiles;
+};
+
+// Range of the (tile, k-block) iteration space owned by a CTA.
+__device__ __forceinline__ void mega_range(const MegaGemmShape& gs, int cta, long long& it0, long long& it1) {
+  if (cta < gs.gsplit) {
+    it0 = (long long)cta * gs.total / gs.gsplit;
+    it1 = (long long)(cta + 1) * gs.total / gs.gsplit;
+  } else {
+    it0 = it1 = 0;
+  }
+}
+
+struct MegaArgs {
+  // model
+  int n_layers, d, H, Dh, F, V, eos_id;
+  float eps;
+  const uint8_t* const* wptr;      // [4*L + 1] tiled weights in execution order (qkv, o, gate/up, down)*L, lm head
+  const bf16* const* norm_ptr;     // [2*L + 1] gains: attn_norm(l), ffn_norm(l) ..., final
+  const bf16* embed;
+  const float* inv_freq;
+  MegaGemmShape shape[5];          // qkv, o, gate/up, down, lm head
+  // batch
+  int B, NT, stages, tmem_cols;
+  RowState st;
+  KvLayout kv;
+  // activations (decode buffers)
+  float* h;                        // [B][d] residual stream
+  bf16 *x, *o, *act;               // GEMM operands: x' [B][d], attention out [B][d], SwiGLU out [B][F]
+  float* rowss;                    // [B][kMaxSlices] sums of squares of h per slice
+  float* partial;
+  float *part_ml, *part_acc;       // attention partials [B][H][max_chunks][2 | Dh]
+  int32_t* attn_count;             // [B][H] arrival counters (zero between uses)
+  int max_chunks;                  // per row, in units of kMegaAttnChunk
+  float* tile_val;
+  int32_t* tile_idx;
+  int n_tiles_lm;
+  // options
+  const int32_t* forced;
+  int32_t* next_tokens;
+  float *dump_logits, *dump_hidden;
+  // sync
+  unsigned long long* grid_ctr;    // monotone arrival counter
+  unsigned long long grid_base;    // its value when this launch starts
+  uint32_t* status;
+};
+
+struct MegaSmem {
+  uint64_t full[kGemmMaxStages];
+  uint64_t empty[kGemmMaxStages];
+  uint64_t acc_full[2];
+  uint64_t acc_empty[2];
+  uint32_t tmem_base;
+  volatile int w_issued;           // ring iterations armed by the weight producer
+  volatile int act_epoch;          // projections whose activation operand is complete
+  volatile int abort;
+  int prefix[kMaxBatch + 1];
+  float q_s[8][128];               // per worker warp: rotated query
+  float red[8];
+  uint32_t am_key[2][4][64];       // per-tile arg-max scratch: [tile half][warp][batch row]
+  int am_id[2][4][64];
+};
+
+__device__ __forceinline__ void named_bar_workers() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+__device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
+  unsigned long long v;
+  asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+
+// mbarrier wait that also gives up when the CTA aborts.
+__device__ __forceinline__ bool mega_wait(uint32_t bar, uint32_t parity, MegaSmem* sm, uint32_t* status, uint32_t code) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (sm->abort) return false;
+    if (clock64() - t0 > 4000000000LL) {
+      atomicCAS(status, 0u, code);
+      sm->abort = 1;
+      return false;
+    }
+  }
+}
+
+// Workers only.  Returns false if the CTA aborted.
+__device__ __forceinline__ bool grid_barrier(const MegaArgs& a, MegaSmem* sm, unsigned long long& epoch, int wtid) {
+  fence_proxy_async_all();                 // activations written here are read by TMA elsewhere
+  named_bar_workers();
+  ++epoch;
+  if (wtid == 0) {
+    __threadfence();
+    atomicAdd(a.grid_ctr, 1ULL);
+    const unsigned long long target = a.grid_base + epoch * gridDim.x;
+    const long long t0 = clock64();
+    while (ld_acquire_u64(a.grid_ctr) < target) {
+      if (sm->abort) break;
+      if (clock64() - t0 > 4000000000LL) {
+        atomicCAS(a.status, 0u, (uint32_t)kStatusGridBarrierTimeout);
+        sm->abort = 1;
+        break;
+      }
+    }
+    __threadfence();
+  }
+  named_bar_workers();
+  return sm->abort == 0;
+}
+
+// Sum of the partials of output row n for token tok (CTA order), read past L1.
+__device__ __forceinline__ float sum_partials_cg(const float* __restrict__ partial, const MegaGemmShape& s, int NT, int n, int tok) {
+  const int4 t = __ldg(reinterpret_cast<const int4*>(s.tiles) + (n >> 7));
+  const size_t slot_stride = (size_t)NT * 128;
+  const size_t off = (size_t)tok * 128 + (n & 127);
+  float acc = __ldcg(partial + (size_t)t.x * slot_stride + off);
+  const size_t cta_stride = slot_stride * s.max_seg;
+  for (int c = t.y; c <= t.z; ++c) acc += __ldcg(partial + (size_t)c * cta_stride + off);
+  return acc;
+}
+
+__device__ __forceinline__ float row_inv_rms(const MegaArgs& a, int r) {
+  const int ns = (a.d + kRowSlice - 1) / kRowSlice;
+  float ss = 0.f;
+  for (int s = 0; s < ns; ++s) ss += __ldcg(a.rowss + (size_t)r * kMaxSlices + s);
+  return rsqrtf(ss / a.d + a.eps);
+}
+
+// ---- stage: embedding (or residual add) + lazy RMSNorm operand -------------------------------------
+// Work item = (row, slice of kRowSlice elements), dealt to CTAs; 256 worker threads, 2 elements each.
+// mode 0: h = E[cur_tok]; mode 1: h += projection (partials of shape `gs`).
+__device__ void stage_residual(const MegaArgs& a, MegaSmem* sm, int wtid, int mode, const MegaGemmShape* gs,
+                               const bf16* __restrict__ gain, bool dump) {
+  const int ns = (a.d + kRowSlice - 1) / kRowSlice;
+  const int n_items = a.B * ns;
+  const int lane = wtid & 31, wid = wtid >> 5;
+  for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
+    const int r = item / ns, sl = item - r * ns;
+    float ss = 0.f;
+    if (a.st.active[r]) {
+      int tok = 0;
+      if (mode == 0) {
+        tok = a.st.cur_tok[r];
+        if (tok < 0 || tok >= a.V) tok = 0;
+      }
+#pragma unroll
+      for (int j = 0; j < kRowSlice / kMegaWorkers; ++j) {
+        const int i = sl * kRowSlice + wtid + j * kMegaWorkers;
+        if (i < a.d) {
+          float v;
+          if (mode == 0) v = __bfloat162float(a.embed[(size_t)tok * a.d + i]);
+          else v = __ldcg(a.h + (size_t)r * a.d + i) + sum_partials_cg(a.partial, *gs, a.NT, i, r);
+          a.h[(size_t)r * a.d + i] = v;
+          if (dump && a.dump_hidden) a.dump_hidden[(size_t)r * a.d + i] = v;
+          a.x[(size_t)r * a.d + i] = __float2bfloat16_rn(v * __bfloat162float(gain[i]));
+          ss += v * v;
+        }
+      }
+    }
+    ss = warp_sum(ss);
+    named_bar_workers();
+    if (lane == 0) sm->red[wid] = ss;
+    named_bar_workers();
+    if (wtid == 0 && a.st.active[r]) {
+      float t = 0.f;
+#pragma unroll
+      for (int w = 0; w < 8; ++w) t += sm->red[w];
+      a.rowss[(size_t)r * kMaxSlices + sl] = t;
+    }
+  }
+}
+
+// ---- stage: q,k,v from partials + RoPE + cache append + paged attention + chunk merge -------------------
+// Work item = (row, head, chunk of kMegaAttnChunk cached tokens), one warp each.  The warp of the chunk that
+// holds the new position also builds k,v of the new token, appends them and attends to them from registers.
+// The last warp to finish a (row, head) merges its chunks and writes the bf16 attention output.
+template <int DH>
+__device__ void stage_attention(const MegaArgs& a, MegaSmem* sm, int wtid, int layer) {
+  constexpr int EPL = DH / 32;             // elements per lane in the "lane + 32 j" layout
+  constexpr int GROUP = DH / 8;            // lanes per key in the 8-elements-per-lane layout
+  constexpr int KPW = 32 / GROUP;          // keys per warp-wide load
+  constexpr int half = DH / 2;
+  const int lane = wtid & 31, wid = wtid >> 5;
+  const int B = a.B, H = a.H, d = a.d;
+  const MegaGemmShape& gs = a.shape[0];
+  // exclusive prefix of chunk counts over rows
+  if (wid == 0) {
+    int cnt[8], loc = 0;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const int r = lane * 8 + j;
+      int c = 0;
+      if (r < B && a.st.active[r]) c = (a.st.ctx_len[r] + 1 + kMegaAttnChunk - 1) / kMegaAttnChunk;
+      cnt[j] = c;
+      loc += c;
+    }
+    int inc = loc;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += t;
+    }
+    int run = inc - loc;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      sm->prefix[lane * 8 + j] = run;
+      run += cnt[j];
+    }
+    if (lane == 31) sm->prefix[kMaxBatch] = inc;
+  }
+  named_bar_workers();
+  const int n_items = sm->prefix[kMaxBatch] * H;
+  const int gl = lane % GROUP, g = lane / GROUP;
+  const float qscale = rsqrtf((float)DH) * 1.4426950408889634f;
+  const bf16* kv_layer = a.kv.pool + (size_t)layer * a.kv.layer_stride;
+  const size_t v_off = (size_t)H * kPageTokens * DH;
+  float* qs = sm->q_s[wid];
+
+  for (int item = blockIdx.x * 8 + wid; item < n_items; item += gridDim.x * 8) {
+    const int cidx = item / H, hd = item - cidx * H;
+    int lo = 0, hi = B - 1;
+    while (lo < hi) {
+      const int mid = (lo + hi + 1) >> 1;
+      if (sm->prefix[mid] <= cidx) lo = mid; else hi = mid - 1;
+    }
+    const int r = lo, chunk = cidx - sm->prefix[r];
+    const int pos = a.st.ctx_len[r];                 // position of the new token; cached tokens are 0..pos-1
+    const int nch = (pos + 1 + kMegaAttnChunk - 1) / kMegaAttnChunk;
+    const int t0 = chunk * kMegaAttnChunk;
+    const int t1 = min(t0 + kMegaAttnChunk, pos);    // cached tokens of this chunk: [t0, t1)
+    const bool has_new = (chunk == nch - 1);
+    const float inv = row_inv_rms(a, r);
+
+    // q in the lane + 32 j layout, RoPE, rounded to bf16 as the operand the attention uses
+    float qv[EPL], sn[EPL / 2 > 0 ? EPL / 2 : 1], cs[EPL / 2 > 0 ? EPL / 2 : 1];
+#pragma unroll
+    for (int j = 0; j < EPL; ++j) qv[j] = inv * sum_partials_cg(a.partial, gs, a.NT, hd * DH + lane + 32 * j, r);
+    // element lane + 32 j pairs with lane + 32 (j + EPL/2); both live in this lane; frequency index lane + 32 j
+#pragma unroll
+    for (int j = 0; j < EPL / 2; ++j) sincosf((float)pos * a.inv_freq[lane + 32 * j], &sn[j], &cs[j]);
+    __syncwarp();
+#pragma unroll
+    for (int j = 0; j < EPL / 2; ++j) {
+      const float x0 = qv[j], x1 = qv[j + EPL / 2];
+      qs[lane + 32 * j] = __bfloat162float(__float2bfloat16_rn(x0 * cs[j] - x1 * sn[j])) * qscale;
+      qs[lane + 32 * j + half] = __bfloat162float(__float2bfloat16_rn(x1 * cs[j] + x0 * sn[j])) * qscale;
+    }
+    __syncwarp();
+    float q[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) q[j] = qs[gl * 8 + j];
+
+    float m = -CUDART_INF_F, l = 0.f, acc[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+
+    // cached tokens, KPW keys per load, 4 loads in flight per lane
+    constexpr int U = 4;
+    for (int base = t0; base < t1; base += KPW * U) {
+      uint4 kk[U], vv[U];
+      bool valid[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int t = base + u * KPW + g;
+        valid[u] = t < t1;
+        kk[u] = make_uint4(0, 0, 0, 0);
+        vv[u] = kk[u];
+        if (valid[u]) {
+          int pg = a.st.block_table[(size_t)r * a.st.max_pages + t / kPageTokens];
+          if (pg < 0 || pg >= a.kv.n_pages) { atomicCAS(a.status, 0u, (uint32_t)kStatusBadPage); pg = 0; }
+          const bf16* kp = kv_layer + (size_t)pg * a.kv.page_elems + ((size_t)hd * kPageTokens + (t % kPageTokens)) * DH + gl * 8;
+          kk[u] = __ldg(reinterpret_cast<const uint4*>(kp));
+          vv[u] = __ldg(reinterpret_cast<const uint4*>(kp + v_off));
+        }
+      }
+      float s[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        float kf[8], dot = 0.f;
+        unpack8(kk[u], kf);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) dot += q[j] * kf[j];
+#pragma unroll
+        for (int o = GROUP / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+        s[u] = valid[u] ? dot : -CUDART_INF_F;
+      }
+      float mn = m;
+#pragma unroll
+      for (int u = 0; u < U; ++u) mn = fmaxf(mn, s[u]);
+      const float sc = (mn == -CUDART_INF_F) ? 1.f : exp2f(m - mn);
+      l *= sc;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) acc[j] *= sc;
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        if (valid[u]) {
+          const float pw = exp2f(s[u] - mn);
+          float vf[8];
+          unpack8(vv[u], vf);
+          l += pw;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) acc[j] += pw * vf[j];
+        }
+      }
+      m = mn;
+    }
+
+    if (has_new) {
+      // k, v of the new token: from partials, RoPE on k, bf16, append to the page, attend from registers
+      float kvv[EPL], vvv[EPL];
+#pragma unroll
+      for (int j = 0; j < EPL; ++j) {
+        kvv[j] = inv * sum_partials_cg(a.partial, gs, a.NT, d + hd * DH + lane + 32 * j, r);
+        vvv[j] = inv * sum_partials_cg(a.partial, gs, a.NT, 2 * d + hd * DH + lane + 32 * j, r);
+      }
+      int pg = a.st.block_table[(size_t)r * a.st.max_pages + pos / kPageTokens];
+      if (pg < 0 || pg >= a.kv.n_pages) { atomicCAS(a.status, 0u, (uint32_t)kStatusBadPage); pg = -1; }
+      bf16* kbase = a.kv.pool + (size_t)layer * a.kv.layer_stride + (size_t)(pg < 0 ? 0 : pg) * a.kv.page_elems +
+                    ((size_t)hd * kPageTokens + (pos % kPageTokens)) * DH;
+      bf16* vbase = kbase + v_off;
+      float dotn = 0.f;
+      float vb[EPL];
+#pragma unroll
+      for (int j = 0; j < EPL / 2; ++j) {
+        const bf16 k0 = __float2bfloat16_rn(kvv[j] * cs[j] - kvv[j + EPL / 2] * sn[j]);
+        const bf16 k1 = __float2bfloat16_rn(kvv[j + EPL / 2] * cs[j] + kvv[j] * sn[j]);
+        const bf16 v0 = __float2bfloat16_rn(vvv[j]), v1 = __float2bfloat16_rn(vvv[j + EPL / 2]);
+        if (pg >= 0) {
+          kbase[lane + 32 * j] = k0;
+          kbase[lane + 32 * j + half] = k1;
+          vbase[lane + 32 * j] = v0;
+          vbase[lane + 32 * j + half] = v1;
+        }
+        dotn += qs[lane + 32 * j] * __bfloat162float(k0) + qs[lane + 32 * j + half] * __bfloat162float(k1);
+        vb[j] = __bfloat162float(v0);
+        vb[j + EPL / 2] = __bfloat162float(v1);
+      }
+      dotn = warp_sum(dotn);
+      // move v of the new token into the 8-per-lane layout through shared memory (q is no longer needed there)
+      __syncwarp();
+#pragma unroll
+      for (int j = 0; j < EPL / 2; ++j) {
+        qs[lane + 32 * j] = vb[j];
+        qs[lane + 32 * j + half] = vb[j + EPL / 2];
+      }
+      __syncwarp();
+      if (g == 0) {                      // key group 0 takes the new token
+        const float mn = fmaxf(m, dotn);
+        const float sc = (m == -CUDART_INF_F) ? 0.f : exp2f(m - mn);
+        const float pw = exp2f(dotn - mn);
+        l = l * sc + pw;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[j] = acc[j] * sc + pw * qs[gl * 8 + j];
+        m = mn;
+      }
+      __syncwarp();
+    }
+
+    // merge the KPW key groups of the warp (same gl, different g): xor over the group index bits
+#pragma unroll
+    for (int o = GROUP; o < 32; o <<= 1) {
+      const float om = __shfl_xor_sync(0xffffffffu, m, o);
+      const float ol = __shfl_xor_sync(0xffffffffu, l, o);
+      const float mn = fmaxf(m, om);
+      const float w0 = (m == -CUDART_INF_F) ? 0.f : exp2f(m - mn);
+      const float w1 = (om == -CUDART_INF_F) ? 0.f : exp2f(om - mn);
+      l = l * w0 + ol * w1;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const float oa = __shfl_xor_sync(0xffffffffu, acc[j], o);
+        acc[j] = acc[j] * w0 + oa * w1;
+      }
+      m = mn;
+    }
+
+    if (nch == 1) {
+      // the only chunk of its (row, head): write the output directly
+      if (g == 0) {
+        const float il = 1.f / l;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) a.o[(size_t)r * d + hd * DH + gl * 8 + j] = __float2bfloat16_rn(acc[j] * il);
+      }
+    } else {
+      const size_t slot = ((size_t)r * H + hd) * a.max_chunks + chunk;
+      if (g == 0) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) a.part_acc[slot * DH + gl * 8 + j] = acc[j];
+        if (gl == 0) { a.part_ml[slot * 2] = m; a.part_ml[slot * 2 + 1] = l; }
+      }
+      __threadfence();
+      __syncwarp();
+      int prev = 0;
+      if (lane == 0) prev = atomicAdd(a.attn_count + r * H + hd, 1);
+      prev = __shfl_sync(0xffffffffu, prev, 0);
+      if (prev == nch - 1) {
+        __threadfence();
+        const size_t base = ((size_t)r * H + hd) * a.max_chunks;
+        float M = -CUDART_INF_F;
+        for (int c = 0; c < nch; ++c) M = fmaxf(M, __ldcg(a.part_ml + (base + c) * 2));
+        float L = 0.f, A[EPL];
+#pragma unroll
+        for (int j = 0; j < EPL; ++j) A[j] = 0.f;
+        for (int c = 0; c < nch; ++c) {
+          const float w = exp2f(__ldcg(a.part_ml + (base + c) * 2) - M);
+          L += __ldcg(a.part_ml + (base + c) * 2 + 1) * w;
+#pragma unroll
+          for (int j = 0; j < EPL; ++j) A[j] += __ldcg(a.part_acc + (base + c) * DH + lane + 32 * j) * w;
+        }
+        const float il = 1.f / L;
+#pragma unroll
+        for (int j = 0; j < EPL; ++j) a.o[(size_t)r * d + hd * DH + lane + 32 * j] = __float2bfloat16_rn(A[j] * il);
+        if (lane == 0) a.attn_count[r * H + hd] = 0;
+      }
+    }
+    __syncwarp();
+  }
+}
+
+// ---- stage: SwiGLU ----------------------------------------------------------------------------------
+__device__ void stage_swiglu(const MegaArgs& a, int wtid) {
+  const MegaGemmShape& gs = a.shape[2];
+  const long long n = (long long)a.B * a.F;
+  for (long long e = (long long)blockIdx.x * kMegaWorkers + wtid; e < n; e += (long long)gridDim.x * kMegaWorkers) {
+    const int r = (int)(e / a.F), f = (int)(e - (long long)r * a.F);
+    if (!a.st.active[r]) continue;
+    const float inv = row_inv_rms(a, r);
+    const float gt = inv * sum_partials_cg(a.partial, gs, a.NT, f, r);
+    const float up = inv * sum_partials_cg(a.partial, gs, a.NT, a.F + f, r);
+    a.act[(size_t)r * a.F + f] = __float2bfloat16_rn(gt / (1.f + __expf(-gt)) * up);
+  }
+}
+
+// ---- stage: per-tile arg-max of the logits --------------------------------------------------------------
+// One vocabulary tile per half of the workers (128 threads = the tile's rows).
+__device__ void stage_tile_argmax(const MegaArgs& a, MegaSmem* sm, int wtid) {
+  const MegaGemmShape& gs = a.shape[4];
+  const int half_id = wtid >> 7, t128 = wtid & 127, lane = wtid & 31, w4 = t128 >> 5;
+  uint32_t* s_key = &sm->am_key[half_id][0][0];       // [4 warps][64 batch rows]
+  int* s_id = &sm->am_id[half_id][0][0];
+  for (int tile0 = blockIdx.x * 2; tile0 < a.n_tiles_lm; tile0 += gridDim.x * 2) {
+    const int tile = tile0 + half_id;
+    const bool tile_ok = tile < a.n_tiles_lm;
+    const int v = tile * 128 + t128;
+    for (int rb = 0; rb < a.B; rb += 64) {              // 64 batch rows at a time (scratch holds 4 x 64 per half)
+      const int rend = min(a.B, rb + 64);
+      for (int r = rb; r < rend; ++r) {
+        uint32_t key = 0;
+        if (tile_ok && a.st.active[r]) {
+          if (v < a.V) {
+            const float lg = row_inv_rms(a, r) * sum_partials_cg(a.partial, gs, a.NT, v, r);
+            if (a.dump_logits) a.dump_logits[(size_t)r * a.V + v] = lg;
+            if (!(a.st.eos_at[r] > 0 && v == a.eos_id)) key = float_order_key(lg);
+          }
+        }
+        const uint32_t best = __reduce_max_sync(0xffffffffu, key);
+        const uint32_t who = __ballot_sync(0xffffffffu, key == best);
+        if (lane == 0) {
+          s_key[w4 * 64 + (r - rb)] = best;
+          s_id[w4 * 64 + (r - rb)] = tile * 128 + w4 * 32 + (__ffs(who) - 1);
+        }
+      }
+      named_bar_workers();
+      if (tile_ok) {
+        for (int r = rb + t128; r < rend; r += 128) {
+          if (!a.st.active[r]) continue;
+          uint32_t bk = s_key[r - rb];
+          int bi = s_id[r - rb];
+#pragma unroll
+          for (int w = 1; w < 4; ++w)
+            if (s_key[w * 64 + (r - rb)] > bk) { bk = s_key[w * 64 + (r - rb)]; bi = s_id[w * 64 + (r - rb)]; }
+          a.tile_val[(size_t)r * a.n_tiles_lm + tile] = __uint_as_float(bk);
+          a.tile_idx[(size_t)r * a.n_tiles_lm + tile] = bi;
+        }
+      }
+      named_bar_workers();
+    }
+  }
+}
+
+// ---- stage: final arg-max over tiles + row bookkeeping (one warp per row) -------------------------------
+__device__ void stage_final(const MegaArgs& a, int wtid) {
+  const int lane = wtid & 31, wid = wtid >> 5;
+  for (int r = blockIdx.x * 8 + wid; r < a.B; r += gridDim.x * 8) {
+    int tok = a.eos_id;
+    if (a.st.active[r]) {
+      uint32_t bk = 0;
+      int bi = 0x7fffffff;
+      for (int t = lane; t < a.n_tiles_lm; t += 32) {
+        const uint32_t k = __float_as_uint(__ldcg(a.tile_val + (size_t)r * a.n_tiles_lm + t));
+        const int id = __ldcg(a.tile_idx + (size_t)r * a.n_tiles_lm + t);
+        if (k > bk || (k == bk && id < bi)) { bk = k; bi = id; }
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        const uint32_t ok = __shfl_xor_sync(0xffffffffu, bk, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+        if (ok > bk || (ok == bk && oi < bi)) { bk = ok; bi = oi; }
+      }
+      if (lane == 0) {
+        a.st.ctx_len[r] += 1;
+        const int cap = a.st.scalars[0];
+        const int gidx = a.st.gen[r] + 1;
+        tok = (bi == 0x7fffffff) ? 0 : bi;
+        if (a.st.eos_at[r] > 0 && gidx == a.st.eos_at[r]) tok = a.eos_id;
+        if (a.forced) tok = a.forced[r];
+        a.st.out_tokens[(size_t)r * a.st.max_new + (gidx - 1)] = tok;
+        a.st.gen[r] = gidx;
+        a.st.cur_tok[r] = tok;
+        if (tok == a.eos_id) { a.st.finished[r] = 1; a.st.active[r] = 0; }
+        else if (gidx >= cap) { a.st.active[r] = 0; }
+        else atomicAdd(a.st.scalars + 1, 1);
+      }
+    }
+    if (lane == 0 && a.next_tokens) a.next_tokens[r] = tok;
+  }
+}
+
+// ------------------------------------------------------------------------------------ the kernel
+template <int DH>
+__global__ void __launch_bounds__(kMegaThreads, 1)
+decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_o,
+                        const __grid_constant__ CUtensorMap map_act, const __grid_constant__ MegaArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  MegaSmem* sm = reinterpret_cast<MegaSmem*>(smem_raw);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int cta = blockIdx.x, G = gridDim.x;
+  const uint32_t stage0 = (smem_u32(smem_raw) + (uint32_t)sizeof(MegaSmem) + 1023u) & ~1023u;
+  const uint32_t a_bytes = kTileM * kTileK * 2;
+  const uint32_t b_bytes = (uint32_t)a.NT * kTileK * 2;
+  const uint32_t stage_bytes = a_bytes + b_bytes;
+  const int S = a.stages;
+  const int n_gemm = 4 * a.n_layers + 1;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < S; ++s) {
+      mbar_init(smem_u32(&sm->full[s]), 1);
+      mbar_init(smem_u32(&sm->empty[s]), 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&sm->acc_full[b]), 1);
+      mbar_init(smem_u32(&sm->acc_empty[b]), 8);
+    }
+    sm->w_issued = 0;
+    sm->act_epoch = 0;
+    sm->abort = 0;
+    fence_barrier_init();
+    tma_prefetch_desc(&map_x);
+    tma_prefetch_desc(&map_o);
+    tma_prefetch_desc(&map_act);
+  }
+  if (warp == 1) {
+    tmem_alloc(smem_u32(&sm->tmem_base), (uint32_t)a.tmem_cols);
+    tmem_relinquish();
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = sm->tmem_base;
+
+  if (warp == 0) {
+    // ===================== weight producer =====================
+    if (lane == 0) {
+      uint64_t hint_w;
+      asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(hint_w));
+      int gi = 0;
+      bool ok = true;
+      for (int gm = 0; gm < n_gemm && ok; ++gm) {
+        const MegaGemmShape& gs = a.shape[gm == n_gemm - 1 ? 4 : (gm & 3)];
+        const uint8_t* w = a.wptr[gm];
+        long long it0, it1;
+        mega_range(gs, cta, it0, it1);
+        for (long long it = it0; it < it1; ++it, ++gi) {
+          const int stage = gi % S;
+          if (gi >= S) {
+            ok = mega_wait(smem_u32(&sm->empty[stage]), (uint32_t)(((gi / S) & 1) ^ 1), sm, a.status, kStatusProducerTimeout);
+            if (!ok) break;
+          }
+          const uint32_t full = smem_u32(&sm->full[stage]);
+          mbar_expect_tx(full, stage_bytes);
+          bulk_load(stage0 + stage * stage_bytes, w + (size_t)it * a_bytes, a_bytes, full, hint_w);
+          __threadfence_block();
+          sm->w_issued = gi + 1;
+        }
+      }
+    }
+  } else if (warp == 2) {
+    // ===================== activation loader =====================
+    if (lane == 0) {
+      uint64_t hint_x;
+      asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(hint_x));
+      int gi = 0;
+      bool ok = true;
+      for (int gm = 0; gm < n_gemm && ok; ++gm) {
+        const int type = gm == n_gemm - 1 ? 4 : (gm & 3);
+        const MegaGemmShape& gs = a.shape[type];
+        const CUtensorMap* mp = (type == 1) ? &map_o : (type == 3) ? &map_act : &map_x;
+        long long it0, it1;
+        mega_range(gs, cta, it0, it1);
+        if (it0 == it1) continue;
+        // the operand is complete once the workers have passed the grid barrier before this projection
+        {
+          const long long t0 = clock64();
+          while (sm->act_epoch <= gm) {
+            if (sm->abort) { ok = false; break; }
+            if (clock64() - t0 > 4000000000LL) {
+              atomicCAS(a.status, 0u, (uint32_t)kStatusFlagTimeout);
+              sm->abort = 1;
+              ok = false;
+              break;
+            }
+          }
+          if (!ok) break;
+          __threadfence();
+          fence_proxy_async_all();
+        }
+        for (long long it = it0; it < it1; ++it, ++gi) {
+          const long long t0 = clock64();
+          while (sm->w_issued <= gi) {
+            if (sm->abort) { ok = false; break; }
+            if (clock64() - t0 > 4000000000LL) {
+              atomicCAS(a.status, 0u, (uint32_t)kStatusFlagTimeout);
+              sm->abort = 1;
+              ok = false;
+              break;
+            }
+          }
+          if (!ok) break;
+          const int stage = gi % S;
+          tma_load_2d(stage0 + stage * stage_bytes + a_bytes, mp, smem_u32(&sm->full[stage]), (int)(it % gs.kb) * kTileK, 0,
+                      hint_x);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ===================== MMA issuer =====================
+    if (lane == 0) {
+      const uint32_t idesc = umma_idesc_bf16(a.NT);
+      int gi = 0, seg = 0;
+      bool ok = true;
+      for (int gm = 0; gm < n_gemm && ok; ++gm) {
+        const MegaGemmShape& gs = a.shape[gm == n_gemm - 1 ? 4 : (gm & 3)];
+        long long it0, it1;
+        mega_range(gs, cta, it0, it1);
+        long long it = it0;
+        while (it < it1 && ok) {
+          const int tile = (int)(it / gs.kb);
+          long long seg_end = (long long)(tile + 1) * gs.kb;
+          if (seg_end > it1) seg_end = it1;
+          const int buf = seg & 1;
+          ok = mega_wait(smem_u32(&sm->acc_empty[buf]), (uint32_t)(((seg >> 1) & 1) ^ 1), sm, a.status, kStatusMmaTimeout);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t d_tmem = tmem_base + (uint32_t)(buf * a.NT);
+          bool first = true;
+          for (; it < seg_end; ++it, ++gi) {
+            const int stage = gi % S;
+            ok = mega_wait(smem_u32(&sm->full[stage]), (uint32_t)((gi / S) & 1), sm, a.status, kStatusMmaTimeout);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t sa = stage0 + stage * stage_bytes;
+            const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sa + a_bytes);
+#pragma unroll
+            for (int k = 0; k < kTileK / 16; ++k)
+              umma_bf16(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (first && k == 0) ? 0u : 1u);
+            first = false;
+            umma_commit(smem_u32(&sm->empty[stage]));
+          }
+          if (!ok) break;
+          umma_commit(smem_u32(&sm->acc_full[buf]));
+          ++seg;
+        }
+      }
+    }
+  } else if (warp >= 3) {
+    // ===================== workers =====================
+    const int wtid = threadIdx.x - 96;
+    const int wid = wtid >> 5;
+    const int quarter = warp & 3;                   // tensor-memory lane quarter this warp may read
+    const int colhalf = wid >> 2;                   // warps 3-6 take the first half of the token columns
+    const int row = quarter * 32 + lane;
+    unsigned long long epoch = 0;
+    int seg = 0;
+    bool ok = true;
+
+    if (cta == 0 && wtid == 0) a.st.scalars[1] = 0;   // rows still active after this step (counted in the last stage)
+    stage_residual(a, sm, wtid, 0, nullptr, a.norm_ptr[0], a.n_layers == 0);
+    ok = grid_barrier(a, sm, epoch, wtid);
+    if (ok && wtid == 0) sm->act_epoch = 1;
+
+    for (int gm = 0; gm < n_gemm && ok; ++gm) {
+      const int type = gm == n_gemm - 1 ? 4 : (gm & 3);
+      const int layer = gm >> 2;
+      const MegaGemmShape& gs = a.shape[type];
+      // ---- drain this CTA's segments of projection gm into fp32 partials
+      long long it0, it1;
+        mega_range(gs, cta, it0, it1);
+      long long it = it0;
+      int seg_local = 0;
+      while (it < it1 && ok) {
+        const int tile = (int)(it / gs.kb);
+        long long seg_end = (long long)(tile + 1) * gs.kb;
+        if (seg_end > it1) seg_end = it1;
+        const int buf = seg & 1;
+        ok = mega_wait(smem_u32(&sm->acc_full[buf]), (uint32_t)((seg >> 1) & 1), sm, a.status, kStatusEpilogueTimeout);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * a.NT);
+        const size_t slot = (size_t)cta * gs.max_seg + seg_local;
+        float* dst = a.partial + slot * a.NT * 128 + row;
+        const int c0 = colhalf * (a.NT / 2), c1 = c0 + a.NT / 2;
+        for (int c = c0; c < c1; c += 8) {
+          float v[8];
+          tmem_ld8(taddr + c, v);
+#pragma unroll
+          for (int j = 0; j < 8; ++j)
+            if (c + j < a.B) dst[(size_t)(c + j) * 128] = v[j];
+        }
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&sm->acc_empty[buf]));
+        it = seg_end;
+        ++seg;
+        ++seg_local;
+      }
+      if (!ok) break;
+      ok = grid_barrier(a, sm, epoch, wtid);
+      if (!ok) break;
+      // ---- the stage that consumes the projection
+      if (type == 0) {
+        stage_attention<DH>(a, sm, wtid, layer);
+      } else if (type == 1) {
+        stage_residual(a, sm, wtid, 1, &a.shape[1], a.norm_ptr[2 * layer + 1], false);
+      } else if (type == 2) {
+        stage_swiglu(a, wtid);
+      } else if (type == 3) {
+        stage_residual(a, sm, wtid, 1, &a.shape[3], a.norm_ptr[2 * layer + 2], layer + 1 == a.n_layers);
+      } else {
+        stage_tile_argmax(a, sm, wtid);
+      }
+      ok = grid_barrier(a, sm, epoch, wtid);
+      if (!ok) break;
+      if (type == 4) stage_final(a, wtid);
+      else if (wtid == 0) sm->act_epoch = gm + 2;
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, (uint32_t)a.tmem_cols);
+  }
+}
+
+}  // namespace ss

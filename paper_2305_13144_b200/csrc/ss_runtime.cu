@@ -10,7 +10,7 @@
 #include <string>
 #include <vector>
 
-#include "ss_kernels.cuh"
+#include "ss_decode_mega.cuh"
 
 using namespace ss;
 
@@ -50,7 +50,7 @@ GemmPlan plan_gemm(int n_out, int K, int NT, int tok_tiles, int mode, int n_sm) 
     p.gridx = p.n_tiles;
     p.gridy = tok_tiles;
   }
-  const int ipc = (int)((total + p.gridx - 1) / p.gridx);
+  const int ipc = std::max(1, (int)((total + p.gridx - 1) / p.gridx));
   p.max_seg = (ipc + p.kb - 2) / p.kb + 1;
   const int stage_bytes = kTileM * kTileK * 2 + NT * kTileK * 2;
   const int budget = 227 * 1024 - 2048;                       // header + alignment slack
@@ -129,6 +129,12 @@ struct ss_ctx {
   float *part_ml = nullptr, *part_acc = nullptr;
   int max_chunks = 0;
   TileSeg* tbl[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};   // qkv, o, gate/up, down, lm head
+  float* rowss = nullptr;          // [kMaxBatch][kMaxSlices]
+  int32_t* attn_count = nullptr;   // [kMaxBatch][H]
+  unsigned long long* grid_ctr = nullptr;
+  unsigned long long grid_epochs = 0;   // grid barriers passed by all launches so far
+  const uint8_t** wptr_dev = nullptr;
+  const bf16** norm_dev = nullptr;
   float* tile_val = nullptr;       // [kMaxBatch][n_tiles of the vocabulary]
   int32_t* tile_idx = nullptr;
   int n_tiles_lm = 0;
@@ -252,7 +258,7 @@ struct Offsets {
   std::vector<size_t> attn_norm, wqkv, wo, ffn_norm, wgu, wdown;
   size_t inv_freq, status, rows, block_table, out_tokens, tok, h, x, qkv, attn_o, gu, act;
   size_t h_dec, x_dec, q_dec, o_dec, act_dec, partial, part_ml, part_acc, kv;
-  size_t tbl[5], tile_val, tile_idx;
+  size_t tbl[5], tile_val, tile_idx, rowss, attn_count, grid_ctr, wptr, norm_ptr;
   size_t partial_bytes;
   int R, max_pages, n_pages, max_chunks;
   size_t total;
@@ -318,7 +324,12 @@ void layout(const ss_model_cfg& m, const ss_runtime_cfg& rt, int n_sm, Offsets& 
   }
   o.partial_bytes = pb;
   o.partial = a.take(pb);
-  o.max_chunks = ceil_div(rt.max_ctx, kAttnChunk);
+  o.max_chunks = ceil_div(rt.max_ctx, kMegaAttnChunk);
+  o.rowss = a.take((size_t)kMaxBatch * kMaxSlices * 4);
+  o.attn_count = a.take((size_t)kMaxBatch * m.n_heads * 4);
+  o.grid_ctr = a.take(64);
+  o.wptr = a.take((size_t)(4 * m.n_layers + 1) * sizeof(void*));
+  o.norm_ptr = a.take((size_t)(2 * m.n_layers + 1) * sizeof(void*));
   o.part_ml = a.take((size_t)kMaxBatch * m.n_heads * o.max_chunks * 2 * 4);
   o.part_acc = a.take((size_t)kMaxBatch * m.n_heads * o.max_chunks * m.head_dim * 4);
   for (int i = 0; i < 5; ++i) o.tbl[i] = a.take((size_t)ceil_div(shapes[i][0], kTileM) * sizeof(TileSeg));
@@ -382,61 +393,54 @@ double weight_bytes_per_step(const ss_model_cfg& m) {
 double kv_bytes_per_token(const ss_model_cfg& m) { return 2.0 * m.d_model * 2.0 * m.n_layers; }
 
 // ------------------------------------------------------------------------------------ decode step
+// One cooperative launch of the persistent kernel (see ss_decode_mega.cuh).
 int enqueue_decode_step(ss_ctx* c, const ss_step_opts* opts, int32_t* next_tokens) {
   const ss_model_cfg& m = c->m;
-  const int B = c->B, d = m.d_model, F = m.d_ffn, H = m.n_heads, Dh = m.head_dim, V = m.vocab;
+  const int B = c->B, d = m.d_model, F = m.d_ffn, V = m.vocab;
   const int NT = round_up(B, 16);
   const CUtensorMap *mx, *mo, *ma;
   int rc;
   if ((rc = xmap(c, 3, NT, &mx)) || (rc = xmap(c, 4, NT, &mo)) || (rc = xmap(c, 5, NT, &ma))) return rc;
-  const GemmPlan p_qkv = plan_gemm(3 * d, d, NT, 1, kGemmPartial, c->n_sm);
-  const GemmPlan p_o = plan_gemm(d, d, NT, 1, kGemmPartial, c->n_sm);
-  const GemmPlan p_gu = plan_gemm(2 * F, d, NT, 1, kGemmPartial, c->n_sm);
-  const GemmPlan p_dn = plan_gemm(d, F, NT, 1, kGemmPartial, c->n_sm);
-  const GemmPlan p_lm = plan_gemm(V, d, NT, 1, kGemmPartial, c->n_sm);
-  const bf16* first_norm = m.n_layers ? c->layers[0].attn_norm : c->final_norm;
-  SS_CUDA(c, launch(c, embed_rmsnorm_kernel, dim3(B), dim3(256), 0, (const int32_t*)c->st.cur_tok,
-                    (const int32_t*)c->st.active, (const bf16*)c->embed, first_norm, c->h_dec, c->x_dec, d, m.rms_eps, V));
-  AttnArgs aa{};
-  aa.st = c->st; aa.kv = c->kv; aa.q = c->q_dec; aa.part_ml = c->part_ml; aa.part_acc = c->part_acc;
-  aa.out = c->o_dec; aa.B = B; aa.d = d; aa.max_chunks = c->max_chunks; aa.status = c->status;
-  const int attn_grid = c->n_sm * 4;
-  for (int l = 0; l < m.n_layers; ++l) {
-    const LayerWeights& w = c->layers[l];
-    if ((rc = run_gemm(c, w.wqkv, *mx, p_qkv, kGemmPartial, B, nullptr, nullptr, 0))) return rc;
-    SS_CUDA(c, launch(c, rope_append_decode_kernel, dim3(H, B), dim3(Dh), 0, (const float*)c->partial,
-                      split_of(p_qkv, c->tbl[0]), c->st, c->kv, l, (const float*)c->inv_freq, c->q_dec, d, c->status));
-    aa.layer = l;
-    if (Dh == 128) {
-      SS_CUDA(c, launch(c, attn_decode_kernel<128>, dim3(attn_grid), dim3(128), 0, aa));
-      SS_CUDA(c, launch(c, attn_combine_kernel<128>, dim3(H, B), dim3(128), 0, aa));
-    } else {
-      SS_CUDA(c, launch(c, attn_decode_kernel<64>, dim3(attn_grid), dim3(128), 0, aa));
-      SS_CUDA(c, launch(c, attn_combine_kernel<64>, dim3(H, B), dim3(64), 0, aa));
-    }
-    if ((rc = run_gemm(c, w.wo, *mo, p_o, kGemmPartial, B, nullptr, nullptr, 0))) return rc;
-    SS_CUDA(c, launch(c, residual_rmsnorm_partial_kernel, dim3(B), dim3(1024), 0, (const float*)c->partial,
-                      split_of(p_o, c->tbl[1]), (const int32_t*)c->st.active, c->h_dec, (const bf16*)w.ffn_norm, c->x_dec,
-                      (float*)nullptr, d, m.rms_eps));
-    if ((rc = run_gemm(c, w.wgu, *mx, p_gu, kGemmPartial, B, nullptr, nullptr, 0))) return rc;
-    SS_CUDA(c, launch(c, swiglu_partial_kernel, dim3(ceil_div(F, 256), B), dim3(256), 0, (const float*)c->partial,
-                      split_of(p_gu, c->tbl[2]), c->act_dec, F));
-    if ((rc = run_gemm(c, w.wdown, *ma, p_dn, kGemmPartial, B, nullptr, nullptr, 0))) return rc;
-    const bool last = l + 1 == m.n_layers;
-    const bf16* next_norm = last ? c->final_norm : c->layers[l + 1].attn_norm;
-    SS_CUDA(c, launch(c, residual_rmsnorm_partial_kernel, dim3(B), dim3(1024), 0, (const float*)c->partial,
-                      split_of(p_dn, c->tbl[3]), (const int32_t*)c->st.active, c->h_dec, next_norm, c->x_dec,
-                      (last && opts) ? opts->dump_hidden : (float*)nullptr, d, m.rms_eps));
+  MegaArgs a{};
+  a.n_layers = m.n_layers; a.d = d; a.H = m.n_heads; a.Dh = m.head_dim; a.F = F; a.V = V; a.eos_id = m.eos_id;
+  a.eps = m.rms_eps;
+  a.wptr = c->wptr_dev;
+  a.norm_ptr = c->norm_dev;
+  a.embed = c->embed;
+  a.inv_freq = c->inv_freq;
+  const int shp[5][2] = {{3 * d, d}, {d, d}, {2 * F, d}, {d, F}, {V, d}};
+  size_t need_partial = 0;
+  for (int i = 0; i < 5; ++i) {
+    const GemmPlan p = plan_gemm(shp[i][0], shp[i][1], NT, 1, kGemmPartial, c->n_sm);
+    a.shape[i] = {p.n_tiles, p.kb, p.max_seg, p.gridx, (long long)p.n_tiles * p.kb, c->tbl[i]};
+    need_partial = std::max(need_partial, (size_t)p.gridx * p.max_seg * NT * 128 * sizeof(float));
   }
-  if (m.n_layers == 0 && opts && opts->dump_hidden)
-    SS_CUDA(c, cudaMemcpyAsync(opts->dump_hidden, c->h_dec, (size_t)B * d * 4, cudaMemcpyDeviceToDevice, c->stream));
-  if ((rc = run_gemm(c, c->lm_head, *mx, p_lm, kGemmPartial, B, nullptr, nullptr, 0))) return rc;
-  SS_CUDA(c, launch(c, lmhead_tile_argmax_kernel, dim3(c->n_tiles_lm), dim3(128), 0, (const float*)c->partial,
-                    split_of(p_lm, c->tbl[4]), c->st, opts ? opts->dump_logits : (float*)nullptr, c->tile_val,
-                    c->tile_idx, B, V, c->n_tiles_lm, m.eos_id));
-  SS_CUDA(c, launch(c, bookkeeping_kernel, dim3(1), dim3(1024), 0, c->st, (const float*)c->tile_val,
-                    (const int32_t*)c->tile_idx, c->n_tiles_lm, opts ? opts->forced_tokens : (const int32_t*)nullptr,
-                    next_tokens, B, m.eos_id, 0));
+  if (need_partial > c->partial_bytes) return SS_ERR_CAPACITY;
+  a.B = B; a.NT = NT;
+  const int stage_bytes = kTileM * kTileK * 2 + NT * kTileK * 2;
+  const int header = (int)sizeof(MegaSmem) + 1024;
+  a.stages = std::max(2, std::min(kGemmMaxStages, (227 * 1024 - header) / stage_bytes));
+  const size_t smem = (size_t)header + (size_t)a.stages * stage_bytes;
+  int cols = 32;
+  while (cols < 2 * NT) cols <<= 1;
+  a.tmem_cols = cols;
+  a.st = c->st; a.kv = c->kv;
+  a.h = c->h_dec; a.x = c->x_dec; a.o = c->o_dec; a.act = c->act_dec;
+  a.rowss = c->rowss; a.partial = c->partial;
+  a.part_ml = c->part_ml; a.part_acc = c->part_acc; a.attn_count = c->attn_count; a.max_chunks = c->max_chunks;
+  a.tile_val = c->tile_val; a.tile_idx = c->tile_idx; a.n_tiles_lm = c->n_tiles_lm;
+  a.forced = opts ? opts->forced_tokens : nullptr;
+  a.next_tokens = next_tokens;
+  a.dump_logits = opts ? opts->dump_logits : nullptr;
+  a.dump_hidden = opts ? opts->dump_hidden : nullptr;
+  a.grid_ctr = c->grid_ctr;
+  a.grid_base = c->grid_epochs * (unsigned long long)c->n_sm;
+  a.status = c->status;
+  void* args[4] = {(void*)mx, (void*)mo, (void*)ma, (void*)&a};
+  const void* fn = m.head_dim == 128 ? (const void*)decode_step_mega_kernel<128> : (const void*)decode_step_mega_kernel<64>;
+  SS_CUDA(c, cudaLaunchCooperativeKernel(fn, dim3(c->n_sm), dim3(kMegaThreads), args, smem, c->stream));
+  c->grid_epochs += 1 + 2 * (unsigned long long)(4 * m.n_layers + 1);
+  c->launches++;
   return SS_OK;
 }
 
@@ -595,6 +599,26 @@ int ss_create(const ss_model_cfg* model, const ss_runtime_cfg* rt, void* dev_are
   c->part_ml = (float*)(A + o.part_ml);
   c->part_acc = (float*)(A + o.part_acc);
   c->max_chunks = o.max_chunks;
+  c->rowss = (float*)(A + o.rowss);
+  c->attn_count = (int32_t*)(A + o.attn_count);
+  c->grid_ctr = (unsigned long long*)(A + o.grid_ctr);
+  c->wptr_dev = (const uint8_t**)(A + o.wptr);
+  c->norm_dev = (const bf16**)(A + o.norm_ptr);
+  {
+    std::vector<const uint8_t*> wp;
+    std::vector<const bf16*> np;
+    for (int l = 0; l < model->n_layers; ++l) {
+      const LayerWeights& w = c->layers[l];
+      wp.push_back(w.wqkv); wp.push_back(w.wo); wp.push_back(w.wgu); wp.push_back(w.wdown);
+      np.push_back(w.attn_norm); np.push_back(w.ffn_norm);
+    }
+    wp.push_back(c->lm_head);
+    np.push_back(c->final_norm);
+    if (cudaMemcpy(c->wptr_dev, wp.data(), wp.size() * sizeof(void*), cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(c->norm_dev, np.data(), np.size() * sizeof(void*), cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemset(A + o.rowss, 0, o.wptr - o.rowss) != cudaSuccess)
+      return fail(SS_ERR_CUDA);
+  }
   c->tile_val = (float*)(A + o.tile_val);
   c->tile_idx = (int32_t*)(A + o.tile_idx);
   c->n_tiles_lm = ceil_div((int)V, kTileM);
@@ -629,6 +653,10 @@ int ss_create(const ss_model_cfg* model, const ss_runtime_cfg* rt, void* dev_are
   if (e == cudaSuccess) e = cudaHostAlloc((void**)&c->pinned, 64, cudaHostAllocDefault);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(gemm_wx_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(decode_step_mega_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(decode_step_mega_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e != cudaSuccess) {
     c->last_cuda = (int)e;
     delete c;
@@ -806,32 +834,9 @@ int ss_decode_step(ss_ctx* c, const ss_step_opts* opts, int32_t* next_tokens, in
 int ss_decode_steps(ss_ctx* c, int32_t n_steps, int32_t* n_active_host) {
   if (!c || n_steps < 0) return SS_ERR_ARG;
   if (!c->in_batch) return SS_ERR_STATE;
-  auto it = c->graphs.find(c->B);
-  if (it == c->graphs.end()) {
-    // make sure every tensor map the step needs exists before capture starts
-    const CUtensorMap* tmp;
-    const int NT = round_up(c->B, 16);
-    int rc;
-    if ((rc = xmap(c, 3, NT, &tmp)) || (rc = xmap(c, 4, NT, &tmp)) || (rc = xmap(c, 5, NT, &tmp))) return rc;
-    cudaGraph_t g = nullptr;
-    SS_CUDA(c, cudaStreamBeginCapture(c->stream, cudaStreamCaptureModeThreadLocal));
-    c->capturing = true;
-    c->capture_count = 0;
-    rc = enqueue_decode_step(c, nullptr, nullptr);
-    c->capturing = false;
-    cudaError_t e = cudaStreamEndCapture(c->stream, &g);
-    if (rc) { if (g) cudaGraphDestroy(g); return rc; }
-    if (e != cudaSuccess) return cuda_fail(c, e);
-    cudaGraphExec_t ge = nullptr;
-    e = cudaGraphInstantiate(&ge, g, 0);
-    cudaGraphDestroy(g);
-    if (e != cudaSuccess) return cuda_fail(c, e);
-    c->graph_nodes = c->capture_count;
-    it = c->graphs.emplace(c->B, ge).first;
-  }
   for (int s = 0; s < n_steps; ++s) {
-    SS_CUDA(c, cudaGraphLaunch(it->second, c->stream));
-    c->launches += c->graph_nodes;
+    int rc = enqueue_decode_step(c, nullptr, nullptr);
+    if (rc) return rc;
   }
   if (n_active_host)
     SS_CUDA(c, cudaMemcpyAsync(n_active_host, c->st.scalars + 1, 4, cudaMemcpyDeviceToHost, c->stream));
@@ -847,7 +852,14 @@ int ss_read_batch(ss_ctx* c, int32_t* out_tokens, int32_t stride, int32_t* out_l
   SS_CUDA(c, cudaMemcpyAsync(fin.data(), c->st.finished, (size_t)B * 4, cudaMemcpyDeviceToHost, c->stream));
   SS_CUDA(c, cudaMemcpyAsync(c->pinned + 1, c->status, 4, cudaMemcpyDeviceToHost, c->stream));
   SS_CUDA(c, cudaStreamSynchronize(c->stream));
-  if (c->pinned[1] != 0) return c->pinned[1] == (int32_t)kStatusBadPage ? SS_ERR_STATE : SS_ERR_DEVICE_TIMEOUT;
+  if (c->pinned[1] != 0) {
+    // an aborted step leaves the grid-barrier counter and the arrival counters in an unknown state
+    cudaMemsetAsync(c->grid_ctr, 0, 8, c->stream);
+    cudaMemsetAsync(c->attn_count, 0, (size_t)kMaxBatch * c->m.n_heads * 4, c->stream);
+    cudaStreamSynchronize(c->stream);
+    c->grid_epochs = 0;
+    return c->pinned[1] == (int32_t)kStatusBadPage ? SS_ERR_STATE : SS_ERR_DEVICE_TIMEOUT;
+  }
   for (int r = 0; r < B; ++r) {
     if (out_tokens && gen[r] > stride) return SS_ERR_CAPACITY;
     out_len[r] = gen[r];
