@@ -232,6 +232,15 @@ int ss_step_model_bytes(const ss_ctx* ctx, const int32_t* ctx_len, const uint8_t
 int ss_logits_noalloc(const float* hidden, const void* norm_gain, const void* lm_head, int32_t n_rows,
                       int32_t d_model, int32_t vocab, float rms_eps, float* logits, void* stream);
 
+/* Tracing (App. D measures per-token time; this shows where one decode step spends it).  Copies the
+ * time stamps (nanoseconds of the GPU's global timer) that CTA 0 took during the LAST decode step:
+ * out[0] start, out[1] first operand ready, then for each projection in execution order
+ * (qkv, o, gate/up, down per layer, LM head) four stamps: own accumulators drained, all partials
+ * visible, own share of the following stage done, stage complete on every SM.
+ * out: host uint64 [cap]; n receives the number of stamps (2 + 4 * (4 * n_layers + 1));
+ * SS_ERR_CAPACITY if cap is smaller.  Synchronises the stream. */
+int ss_step_trace(ss_ctx* ctx, uint64_t* out, int32_t cap, int32_t* n);
+
 const char* ss_strerror(int code);
 /* Last device status word (0 = clean; non-zero = which bounded wait expired). Synchronises. */
 int ss_last_device_status(ss_ctx* ctx, uint32_t* out);

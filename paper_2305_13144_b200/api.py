@@ -23,7 +23,7 @@ EXPORTS = [
     "ss_arena_bytes", "ss_create", "ss_destroy", "ss_load_weights", "ss_schedule", "ss_prefill",
     "ss_decode_step", "ss_decode_steps", "ss_read_batch", "ss_release_batch", "ss_run_group",
     "ss_step_model_bytes", "ss_strerror", "ss_last_device_status", "ss_last_cuda_error", "ss_kernel_launches",
-    "ss_logits_noalloc",
+    "ss_logits_noalloc", "ss_step_trace",
 ]
 
 
@@ -104,6 +104,7 @@ def lib() -> C.CDLL:
         L.ss_run_group.argtypes = [C.c_void_p] * 7 + [C.c_int32] + [C.c_void_p] * 6 + [C.c_int32, C.c_void_p, C.c_void_p]
         L.ss_step_model_bytes.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(C.c_double)]
         L.ss_last_device_status.argtypes = [C.c_void_p, C.POINTER(C.c_uint32)]
+        L.ss_step_trace.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(C.c_int32)]
         L.ss_logits_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                         C.c_float, C.c_void_p, C.c_void_p]
         _lib_handle = L
@@ -301,6 +302,15 @@ def ss_last_device_status(ctx: Ctx) -> int:
     out = C.c_uint32(0)
     _check(lib().ss_last_device_status(ctx.handle, C.byref(out)), "ss_last_device_status", ctx)
     return out.value
+
+
+def ss_step_trace(ctx: Ctx) -> np.ndarray:
+    """Stage-boundary time stamps (ns) of the last decode step, see include/seqsched.h."""
+    n = C.c_int32(0)
+    cap = 2 + 4 * (4 * ctx.model.n_layers + 1)
+    out = np.zeros(cap, dtype=np.uint64)
+    _check(lib().ss_step_trace(ctx.handle, _hp(out), cap, C.byref(n)), "ss_step_trace", ctx)
+    return out[:n.value]
 
 
 def ss_last_cuda_error(ctx: Ctx) -> int:

@@ -85,7 +85,14 @@ struct MegaArgs {
   unsigned long long* grid_ctr;    // monotone arrival counter
   unsigned long long grid_base;    // its value when this launch starts
   uint32_t* status;
+  unsigned long long* trace;       // [2 + 4 * projections] global-timer stamps of CTA 0 (stage boundaries)
 };
+
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
 
 struct MegaSmem {
   uint64_t full[kGemmMaxStages];
@@ -724,10 +731,14 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
     int seg = 0;
     bool ok = true;
 
+    const bool tracer = cta == 0 && wtid == 0 && a.trace != nullptr;
+    int tr = 0;
+    if (tracer) a.trace[tr++] = global_timer_ns();
     if (cta == 0 && wtid == 0) a.st.scalars[1] = 0;   // rows still active after this step (counted in the last stage)
     stage_residual(a, sm, wtid, 0, nullptr, a.norm_ptr[0], a.n_layers == 0);
     ok = grid_barrier(a, sm, epoch, wtid);
     if (ok && wtid == 0) sm->act_epoch = 1;
+    if (tracer) a.trace[tr++] = global_timer_ns();
 
     for (int gm = 0; gm < n_gemm && ok; ++gm) {
       const int type = gm == n_gemm - 1 ? 4 : (gm & 3);
@@ -766,8 +777,10 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
         ++seg_local;
       }
       if (!ok) break;
+      if (tracer) a.trace[tr++] = global_timer_ns();       // this CTA's accumulators drained
       ok = grid_barrier(a, sm, epoch, wtid);
       if (!ok) break;
+      if (tracer) a.trace[tr++] = global_timer_ns();       // every CTA's partials visible
       // ---- the stage that consumes the projection
       if (type == 0) {
         stage_attention<DH>(a, sm, wtid, layer);
@@ -780,8 +793,10 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
       } else {
         stage_tile_argmax(a, sm, wtid);
       }
+      if (tracer) a.trace[tr++] = global_timer_ns();       // this CTA's share of the stage done
       ok = grid_barrier(a, sm, epoch, wtid);
       if (!ok) break;
+      if (tracer) a.trace[tr++] = global_timer_ns();       // stage complete everywhere
       if (type == 4) stage_final(a, wtid);
       else if (wtid == 0) sm->act_epoch = gm + 2;
     }

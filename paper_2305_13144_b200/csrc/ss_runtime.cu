@@ -132,6 +132,8 @@ struct ss_ctx {
   float* rowss = nullptr;          // [kMaxBatch][kMaxSlices]
   int32_t* attn_count = nullptr;   // [kMaxBatch][H]
   unsigned long long* grid_ctr = nullptr;
+  unsigned long long* trace = nullptr;  // stage-boundary time stamps of the last decode step
+  int trace_len = 0;
   unsigned long long grid_epochs = 0;   // grid barriers passed by all launches so far
   const uint8_t** wptr_dev = nullptr;
   const bf16** norm_dev = nullptr;
@@ -258,7 +260,7 @@ struct Offsets {
   std::vector<size_t> attn_norm, wqkv, wo, ffn_norm, wgu, wdown;
   size_t inv_freq, status, rows, block_table, out_tokens, tok, h, x, qkv, attn_o, gu, act;
   size_t h_dec, x_dec, q_dec, o_dec, act_dec, partial, part_ml, part_acc, kv;
-  size_t tbl[5], tile_val, tile_idx, rowss, attn_count, grid_ctr, wptr, norm_ptr;
+  size_t tbl[5], tile_val, tile_idx, rowss, attn_count, grid_ctr, wptr, norm_ptr, trace;
   size_t partial_bytes;
   int R, max_pages, n_pages, max_chunks;
   size_t total;
@@ -330,6 +332,7 @@ void layout(const ss_model_cfg& m, const ss_runtime_cfg& rt, int n_sm, Offsets& 
   o.grid_ctr = a.take(64);
   o.wptr = a.take((size_t)(4 * m.n_layers + 1) * sizeof(void*));
   o.norm_ptr = a.take((size_t)(2 * m.n_layers + 1) * sizeof(void*));
+  o.trace = a.take((size_t)(2 + 4 * (4 * m.n_layers + 1)) * 8);
   o.part_ml = a.take((size_t)kMaxBatch * m.n_heads * o.max_chunks * 2 * 4);
   o.part_acc = a.take((size_t)kMaxBatch * m.n_heads * o.max_chunks * m.head_dim * 4);
   for (int i = 0; i < 5; ++i) o.tbl[i] = a.take((size_t)ceil_div(shapes[i][0], kTileM) * sizeof(TileSeg));
@@ -436,6 +439,7 @@ int enqueue_decode_step(ss_ctx* c, const ss_step_opts* opts, int32_t* next_token
   a.grid_ctr = c->grid_ctr;
   a.grid_base = c->grid_epochs * (unsigned long long)c->n_sm;
   a.status = c->status;
+  a.trace = c->trace;
   void* args[4] = {(void*)mx, (void*)mo, (void*)ma, (void*)&a};
   const void* fn = m.head_dim == 128 ? (const void*)decode_step_mega_kernel<128> : (const void*)decode_step_mega_kernel<64>;
   SS_CUDA(c, cudaLaunchCooperativeKernel(fn, dim3(c->n_sm), dim3(kMegaThreads), args, smem, c->stream));
@@ -603,6 +607,8 @@ int ss_create(const ss_model_cfg* model, const ss_runtime_cfg* rt, void* dev_are
   c->attn_count = (int32_t*)(A + o.attn_count);
   c->grid_ctr = (unsigned long long*)(A + o.grid_ctr);
   c->wptr_dev = (const uint8_t**)(A + o.wptr);
+  c->trace = (unsigned long long*)(A + o.trace);
+  c->trace_len = 2 + 4 * (4 * model->n_layers + 1);
   c->norm_dev = (const bf16**)(A + o.norm_ptr);
   {
     std::vector<const uint8_t*> wp;
@@ -890,6 +896,15 @@ int ss_last_device_status(ss_ctx* c, uint32_t* out) {
   SS_CUDA(c, cudaMemcpyAsync(c->pinned + 1, c->status, 4, cudaMemcpyDeviceToHost, c->stream));
   SS_CUDA(c, cudaStreamSynchronize(c->stream));
   *out = (uint32_t)c->pinned[1];
+  return SS_OK;
+}
+
+int ss_step_trace(ss_ctx* c, uint64_t* out, int32_t cap, int32_t* n) {
+  if (!c || !out || !n) return SS_ERR_ARG;
+  *n = c->trace_len;
+  if (cap < c->trace_len) return SS_ERR_CAPACITY;
+  SS_CUDA(c, cudaMemcpyAsync(out, c->trace, (size_t)c->trace_len * 8, cudaMemcpyDeviceToHost, c->stream));
+  SS_CUDA(c, cudaStreamSynchronize(c->stream));
   return SS_OK;
 }
 
