@@ -74,6 +74,7 @@ struct MegaArgs {
   float *part_ml, *part_acc;       // attention partials [B][H][max_chunks][2 | Dh]
   int32_t* attn_count;             // [B][H] arrival counters (zero between uses)
   int max_chunks;                  // per row, in units of kMegaAttnChunk
+  int attn_wpp;                    // warps of one CTA that share a (row, head) attention item: 1, 2, 4 or 8
   float* tile_val;
   int32_t* tile_idx;
   int n_tiles_lm;
@@ -104,7 +105,8 @@ struct MegaSmem {
   volatile int act_epoch;          // projections whose activation operand is complete
   volatile int abort;
   int prefix[kMaxBatch + 1];
-  float q_s[8][128];               // per worker warp: rotated query
+  float inv_s[kMaxBatch];          // 1/rms of every row for the running stage
+  float att_s[2][8][136];          // attention: per worker warp (acc[Dh], max, sum), double-buffered
   float red[8];
   uint32_t am_key[2][4][64];       // per-tile arg-max scratch: [tile half][warp][batch row]
   int am_id[2][4][64];
@@ -219,193 +221,182 @@ __device__ void stage_residual(const MegaArgs& a, MegaSmem* sm, int wtid, int mo
   }
 }
 
-// ---- stage: q,k,v from partials + RoPE + cache append + paged attention + chunk merge -------------------
-// Work item = (row, head, chunk of kMegaAttnChunk cached tokens), one warp each.  The warp of the chunk that
-// holds the new position also builds k,v of the new token, appends them and attends to them from registers.
-// The last warp to finish a (row, head) merges its chunks and writes the bf16 attention output.
+// ---- helpers shared by the stages ----------------------------------------------------------------------
+// 8 consecutive outputs n0..n0+7 (n0 a multiple of 8, so they share a tile) for token tok, CTA order.
+__device__ __forceinline__ void sum_partials8_cg(const float* __restrict__ partial, const MegaGemmShape& s, int NT, int n0,
+                                                 int tok, float (&x)[8]) {
+  const int4 t = __ldg(reinterpret_cast<const int4*>(s.tiles) + (n0 >> 7));
+  const size_t slot_stride = (size_t)NT * 128;
+  const size_t off = (size_t)tok * 128 + (n0 & 127);
+  const float4* p = reinterpret_cast<const float4*>(partial + (size_t)t.x * slot_stride + off);
+  float4 u = __ldcg(p), v = __ldcg(p + 1);
+  x[0] = u.x; x[1] = u.y; x[2] = u.z; x[3] = u.w; x[4] = v.x; x[5] = v.y; x[6] = v.z; x[7] = v.w;
+  const size_t cta_stride = slot_stride * s.max_seg;
+  for (int c = t.y; c <= t.z; ++c) {
+    p = reinterpret_cast<const float4*>(partial + (size_t)c * cta_stride + off);
+    u = __ldcg(p);
+    v = __ldcg(p + 1);
+    x[0] += u.x; x[1] += u.y; x[2] += u.z; x[3] += u.w; x[4] += v.x; x[5] += v.y; x[6] += v.z; x[7] += v.w;
+  }
+}
+
+// 1/rms of every active row into shared memory (one pass at the start of a consumer stage).
+__device__ __forceinline__ void stage_inv_rms(const MegaArgs& a, MegaSmem* sm, int wtid) {
+  for (int r = wtid; r < a.B; r += kMegaWorkers) sm->inv_s[r] = a.st.active[r] ? row_inv_rms(a, r) : 0.f;
+  named_bar_workers();
+}
+
+__device__ __forceinline__ void group_bar(int id, int threads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
+// ---- stage: q,k,v from partials + RoPE + cache append + paged attention ----------------------------------
+// Work item = (row, head).  A group of `wpp` warps of one CTA shares an item: every warp rebuilds the
+// rotated query (cheap, and it avoids a hand-off), takes every wpp-th page of the row's cache, and
+// leaves its running (max, sum, acc) in shared memory; the group's first warp also builds k,v of
+// the new token, appends them to the page, attends to them from registers and merges the group.
+// A lane owns 8 consecutive head dimensions (one 128-bit load); Dh/8 lanes cover a key.
 template <int DH>
 __device__ void stage_attention(const MegaArgs& a, MegaSmem* sm, int wtid, int layer) {
-  constexpr int EPL = DH / 32;             // elements per lane in the "lane + 32 j" layout
-  constexpr int GROUP = DH / 8;            // lanes per key in the 8-elements-per-lane layout
+  constexpr int GROUP = DH / 8;            // lanes per key
   constexpr int KPW = 32 / GROUP;          // keys per warp-wide load
-  constexpr int half = DH / 2;
+  constexpr int HL = GROUP / 2;            // lanes holding the first half of the head
+  constexpr int U = 8;                     // warp-wide loads in flight (K and V each)
+  constexpr int EPL = DH / 32;
   const int lane = wtid & 31, wid = wtid >> 5;
-  const int B = a.B, H = a.H, d = a.d;
-  const MegaGemmShape& gs = a.shape[0];
-  // exclusive prefix of chunk counts over rows
-  if (wid == 0) {
-    int cnt[8], loc = 0;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const int r = lane * 8 + j;
-      int c = 0;
-      if (r < B && a.st.active[r]) c = (a.st.ctx_len[r] + 1 + kMegaAttnChunk - 1) / kMegaAttnChunk;
-      cnt[j] = c;
-      loc += c;
-    }
-    int inc = loc;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int t = __shfl_up_sync(0xffffffffu, inc, o);
-      if (lane >= o) inc += t;
-    }
-    int run = inc - loc;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      sm->prefix[lane * 8 + j] = run;
-      run += cnt[j];
-    }
-    if (lane == 31) sm->prefix[kMaxBatch] = inc;
-  }
-  named_bar_workers();
-  const int n_items = sm->prefix[kMaxBatch] * H;
   const int gl = lane % GROUP, g = lane / GROUP;
+  const int wpp = a.attn_wpp, grp = wid / wpp, wig = wid - grp * wpp, GP = 8 / wpp;
+  const int H = a.H, d = a.d;
+  const MegaGemmShape& gs = a.shape[0];
   const float qscale = rsqrtf((float)DH) * 1.4426950408889634f;
   const bf16* kv_layer = a.kv.pool + (size_t)layer * a.kv.layer_stride;
   const size_t v_off = (size_t)H * kPageTokens * DH;
-  float* qs = sm->q_s[wid];
+  const int n_pairs = a.B * H;
+  stage_inv_rms(a, sm, wtid);
+  int buf = 0;
 
-  for (int item = blockIdx.x * 8 + wid; item < n_items; item += gridDim.x * 8) {
-    const int cidx = item / H, hd = item - cidx * H;
-    int lo = 0, hi = B - 1;
-    while (lo < hi) {
-      const int mid = (lo + hi + 1) >> 1;
-      if (sm->prefix[mid] <= cidx) lo = mid; else hi = mid - 1;
-    }
-    const int r = lo, chunk = cidx - sm->prefix[r];
-    const int pos = a.st.ctx_len[r];                 // position of the new token; cached tokens are 0..pos-1
-    const int nch = (pos + 1 + kMegaAttnChunk - 1) / kMegaAttnChunk;
-    const int t0 = chunk * kMegaAttnChunk;
-    const int t1 = min(t0 + kMegaAttnChunk, pos);    // cached tokens of this chunk: [t0, t1)
-    const bool has_new = (chunk == nch - 1);
-    const float inv = row_inv_rms(a, r);
+  for (int p = blockIdx.x * GP + grp; p < n_pairs; p += gridDim.x * GP) {
+    const int r = p / H, hd = p - r * H;
+    if (!a.st.active[r]) continue;                   // uniform within the group
+    const int pos = a.st.ctx_len[r];                 // new token's position; cached tokens are 0..pos-1
+    const float inv = sm->inv_s[r];
 
-    // q in the lane + 32 j layout, RoPE, rounded to bf16 as the operand the attention uses
-    float qv[EPL], sn[EPL / 2 > 0 ? EPL / 2 : 1], cs[EPL / 2 > 0 ? EPL / 2 : 1];
+    // rotation angles of this lane's 8 dimensions (index within the half)
+    float sn[8], cs[8];
+    {
+      const int f0 = (gl % HL) * 8;
 #pragma unroll
-    for (int j = 0; j < EPL; ++j) qv[j] = inv * sum_partials_cg(a.partial, gs, a.NT, hd * DH + lane + 32 * j, r);
-    // element lane + 32 j pairs with lane + 32 (j + EPL/2); both live in this lane; frequency index lane + 32 j
-#pragma unroll
-    for (int j = 0; j < EPL / 2; ++j) sincosf((float)pos * a.inv_freq[lane + 32 * j], &sn[j], &cs[j]);
-    __syncwarp();
-#pragma unroll
-    for (int j = 0; j < EPL / 2; ++j) {
-      const float x0 = qv[j], x1 = qv[j + EPL / 2];
-      qs[lane + 32 * j] = __bfloat162float(__float2bfloat16_rn(x0 * cs[j] - x1 * sn[j])) * qscale;
-      qs[lane + 32 * j + half] = __bfloat162float(__float2bfloat16_rn(x1 * cs[j] + x0 * sn[j])) * qscale;
+      for (int j = 0; j < 8; ++j) sincosf((float)pos * a.inv_freq[f0 + j], &sn[j], &cs[j]);
     }
-    __syncwarp();
+    // q: partial sums, lazy norm, RoPE (partner dimension lives HL lanes away), bf16 rounding
     float q[8];
+    {
+      float x[8];
+      sum_partials8_cg(a.partial, gs, a.NT, hd * DH + gl * 8, r, x);
 #pragma unroll
-    for (int j = 0; j < 8; ++j) q[j] = qs[gl * 8 + j];
+      for (int j = 0; j < 8; ++j) {
+        const float xv = x[j] * inv;
+        const float pv = __shfl_xor_sync(0xffffffffu, xv, HL);
+        const float o = (gl < HL) ? xv * cs[j] - pv * sn[j] : xv * cs[j] + pv * sn[j];
+        q[j] = __bfloat162float(__float2bfloat16_rn(o)) * qscale;
+      }
+    }
 
     float m = -CUDART_INF_F, l = 0.f, acc[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) acc[j] = 0.f;
 
-    // cached tokens, KPW keys per load, 4 loads in flight per lane
-    constexpr int U = 4;
-    for (int base = t0; base < t1; base += KPW * U) {
-      uint4 kk[U], vv[U];
-      bool valid[U];
+    const int npg = (pos + kPageTokens - 1) / kPageTokens;
+    for (int pi = wig; pi < npg; pi += wpp) {
+      int pg = a.st.block_table[(size_t)r * a.st.max_pages + pi];
+      if (pg < 0 || pg >= a.kv.n_pages) { atomicCAS(a.status, 0u, (uint32_t)kStatusBadPage); pg = 0; }
+      const int tcount = min(kPageTokens, pos - pi * kPageTokens);
+      const bf16* kb = kv_layer + (size_t)pg * a.kv.page_elems + (size_t)hd * kPageTokens * DH + gl * 8;
+      for (int tb = 0; tb < tcount; tb += KPW * U) {
+        uint4 kk[U], vv[U];
+        bool valid[U];
 #pragma unroll
-      for (int u = 0; u < U; ++u) {
-        const int t = base + u * KPW + g;
-        valid[u] = t < t1;
-        kk[u] = make_uint4(0, 0, 0, 0);
-        vv[u] = kk[u];
-        if (valid[u]) {
-          int pg = a.st.block_table[(size_t)r * a.st.max_pages + t / kPageTokens];
-          if (pg < 0 || pg >= a.kv.n_pages) { atomicCAS(a.status, 0u, (uint32_t)kStatusBadPage); pg = 0; }
-          const bf16* kp = kv_layer + (size_t)pg * a.kv.page_elems + ((size_t)hd * kPageTokens + (t % kPageTokens)) * DH + gl * 8;
-          kk[u] = __ldg(reinterpret_cast<const uint4*>(kp));
-          vv[u] = __ldg(reinterpret_cast<const uint4*>(kp + v_off));
+        for (int u = 0; u < U; ++u) {
+          const int t = tb + u * KPW + g;
+          valid[u] = t < tcount;
+          kk[u] = make_uint4(0, 0, 0, 0);
+          vv[u] = kk[u];
+          if (valid[u]) {
+            kk[u] = __ldg(reinterpret_cast<const uint4*>(kb + (size_t)t * DH));
+            vv[u] = __ldg(reinterpret_cast<const uint4*>(kb + (size_t)t * DH + v_off));
+          }
         }
-      }
-      float s[U];
+        float s[U];
 #pragma unroll
-      for (int u = 0; u < U; ++u) {
-        float kf[8], dot = 0.f;
-        unpack8(kk[u], kf);
+        for (int u = 0; u < U; ++u) {
+          float kf[8], dot = 0.f;
+          unpack8(kk[u], kf);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) dot += q[j] * kf[j];
+          for (int j = 0; j < 8; ++j) dot += q[j] * kf[j];
 #pragma unroll
-        for (int o = GROUP / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-        s[u] = valid[u] ? dot : -CUDART_INF_F;
-      }
-      float mn = m;
-#pragma unroll
-      for (int u = 0; u < U; ++u) mn = fmaxf(mn, s[u]);
-      const float sc = (mn == -CUDART_INF_F) ? 1.f : exp2f(m - mn);
-      l *= sc;
-#pragma unroll
-      for (int j = 0; j < 8; ++j) acc[j] *= sc;
-#pragma unroll
-      for (int u = 0; u < U; ++u) {
-        if (valid[u]) {
-          const float pw = exp2f(s[u] - mn);
-          float vf[8];
-          unpack8(vv[u], vf);
-          l += pw;
-#pragma unroll
-          for (int j = 0; j < 8; ++j) acc[j] += pw * vf[j];
+          for (int o = GROUP / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+          s[u] = valid[u] ? dot : -CUDART_INF_F;
         }
-      }
-      m = mn;
-    }
-
-    if (has_new) {
-      // k, v of the new token: from partials, RoPE on k, bf16, append to the page, attend from registers
-      float kvv[EPL], vvv[EPL];
+        float mn = m;
 #pragma unroll
-      for (int j = 0; j < EPL; ++j) {
-        kvv[j] = inv * sum_partials_cg(a.partial, gs, a.NT, d + hd * DH + lane + 32 * j, r);
-        vvv[j] = inv * sum_partials_cg(a.partial, gs, a.NT, 2 * d + hd * DH + lane + 32 * j, r);
-      }
-      int pg = a.st.block_table[(size_t)r * a.st.max_pages + pos / kPageTokens];
-      if (pg < 0 || pg >= a.kv.n_pages) { atomicCAS(a.status, 0u, (uint32_t)kStatusBadPage); pg = -1; }
-      bf16* kbase = a.kv.pool + (size_t)layer * a.kv.layer_stride + (size_t)(pg < 0 ? 0 : pg) * a.kv.page_elems +
-                    ((size_t)hd * kPageTokens + (pos % kPageTokens)) * DH;
-      bf16* vbase = kbase + v_off;
-      float dotn = 0.f;
-      float vb[EPL];
+        for (int u = 0; u < U; ++u) mn = fmaxf(mn, s[u]);
+        const float sc = (mn == -CUDART_INF_F) ? 1.f : exp2f(m - mn);
+        l *= sc;
 #pragma unroll
-      for (int j = 0; j < EPL / 2; ++j) {
-        const bf16 k0 = __float2bfloat16_rn(kvv[j] * cs[j] - kvv[j + EPL / 2] * sn[j]);
-        const bf16 k1 = __float2bfloat16_rn(kvv[j + EPL / 2] * cs[j] + kvv[j] * sn[j]);
-        const bf16 v0 = __float2bfloat16_rn(vvv[j]), v1 = __float2bfloat16_rn(vvv[j + EPL / 2]);
-        if (pg >= 0) {
-          kbase[lane + 32 * j] = k0;
-          kbase[lane + 32 * j + half] = k1;
-          vbase[lane + 32 * j] = v0;
-          vbase[lane + 32 * j + half] = v1;
+        for (int j = 0; j < 8; ++j) acc[j] *= sc;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+          if (valid[u]) {
+            const float pw = exp2f(s[u] - mn);
+            float vf[8];
+            unpack8(vv[u], vf);
+            l += pw;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) acc[j] += pw * vf[j];
+          }
         }
-        dotn += qs[lane + 32 * j] * __bfloat162float(k0) + qs[lane + 32 * j + half] * __bfloat162float(k1);
-        vb[j] = __bfloat162float(v0);
-        vb[j + EPL / 2] = __bfloat162float(v1);
-      }
-      dotn = warp_sum(dotn);
-      // move v of the new token into the 8-per-lane layout through shared memory (q is no longer needed there)
-      __syncwarp();
-#pragma unroll
-      for (int j = 0; j < EPL / 2; ++j) {
-        qs[lane + 32 * j] = vb[j];
-        qs[lane + 32 * j + half] = vb[j + EPL / 2];
-      }
-      __syncwarp();
-      if (g == 0) {                      // key group 0 takes the new token
-        const float mn = fmaxf(m, dotn);
-        const float sc = (m == -CUDART_INF_F) ? 0.f : exp2f(m - mn);
-        const float pw = exp2f(dotn - mn);
-        l = l * sc + pw;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) acc[j] = acc[j] * sc + pw * qs[gl * 8 + j];
         m = mn;
       }
-      __syncwarp();
     }
 
-    // merge the KPW key groups of the warp (same gl, different g): xor over the group index bits
+    if (wig == 0) {
+      // the new token: k (rotated), v -> bf16 -> page; its score and value straight from registers
+      float kx[8], vx[8];
+      sum_partials8_cg(a.partial, gs, a.NT, d + hd * DH + gl * 8, r, kx);
+      sum_partials8_cg(a.partial, gs, a.NT, 2 * d + hd * DH + gl * 8, r, vx);
+      __align__(16) bf16 kb8[8], vb8[8];
+      float dot = 0.f;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const float xv = kx[j] * inv;
+        const float pv = __shfl_xor_sync(0xffffffffu, xv, HL);
+        const float o = (gl < HL) ? xv * cs[j] - pv * sn[j] : xv * cs[j] + pv * sn[j];
+        kb8[j] = __float2bfloat16_rn(o);
+        vb8[j] = __float2bfloat16_rn(vx[j] * inv);
+        dot += q[j] * __bfloat162float(kb8[j]);
+      }
+#pragma unroll
+      for (int o = GROUP / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+      int pg = a.st.block_table[(size_t)r * a.st.max_pages + pos / kPageTokens];
+      if (pg < 0 || pg >= a.kv.n_pages) { atomicCAS(a.status, 0u, (uint32_t)kStatusBadPage); pg = -1; }
+      if (g == 0) {
+        if (pg >= 0) {
+          bf16* kdst = a.kv.pool + (size_t)layer * a.kv.layer_stride + (size_t)pg * a.kv.page_elems +
+                       ((size_t)hd * kPageTokens + (pos % kPageTokens)) * DH + gl * 8;
+          *reinterpret_cast<uint4*>(kdst) = *reinterpret_cast<const uint4*>(kb8);
+          *reinterpret_cast<uint4*>(kdst + v_off) = *reinterpret_cast<const uint4*>(vb8);
+        }
+        const float mn = fmaxf(m, dot);
+        const float sc = (m == -CUDART_INF_F) ? 0.f : exp2f(m - mn);
+        const float pw = exp2f(dot - mn);
+        l = l * sc + pw;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[j] = acc[j] * sc + pw * __bfloat162float(vb8[j]);
+        m = mn;
+      }
+    }
+
+    // merge the KPW key groups of the warp (same gl, different g)
 #pragma unroll
     for (int o = GROUP; o < 32; o <<= 1) {
       const float om = __shfl_xor_sync(0xffffffffu, m, o);
@@ -422,60 +413,66 @@ __device__ void stage_attention(const MegaArgs& a, MegaSmem* sm, int wtid, int l
       m = mn;
     }
 
-    if (nch == 1) {
-      // the only chunk of its (row, head): write the output directly
+    if (wpp == 1) {
       if (g == 0) {
         const float il = 1.f / l;
+        __align__(16) bf16 ob[8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) a.o[(size_t)r * d + hd * DH + gl * 8 + j] = __float2bfloat16_rn(acc[j] * il);
+        for (int j = 0; j < 8; ++j) ob[j] = __float2bfloat16_rn(acc[j] * il);
+        *reinterpret_cast<uint4*>(a.o + (size_t)r * d + hd * DH + gl * 8) = *reinterpret_cast<const uint4*>(ob);
       }
     } else {
-      const size_t slot = ((size_t)r * H + hd) * a.max_chunks + chunk;
+      float* slot = sm->att_s[buf][wid];
       if (g == 0) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) a.part_acc[slot * DH + gl * 8 + j] = acc[j];
-        if (gl == 0) { a.part_ml[slot * 2] = m; a.part_ml[slot * 2 + 1] = l; }
+        for (int j = 0; j < 8; ++j) slot[gl * 8 + j] = acc[j];
+        if (gl == 0) { slot[DH] = m; slot[DH + 1] = l; }
       }
-      __threadfence();
-      __syncwarp();
-      int prev = 0;
-      if (lane == 0) prev = atomicAdd(a.attn_count + r * H + hd, 1);
-      prev = __shfl_sync(0xffffffffu, prev, 0);
-      if (prev == nch - 1) {
-        __threadfence();
-        const size_t base = ((size_t)r * H + hd) * a.max_chunks;
+      group_bar(2 + grp, wpp * 32);
+      if (wig == 0) {
+        const int w0i = grp * wpp;
         float M = -CUDART_INF_F;
-        for (int c = 0; c < nch; ++c) M = fmaxf(M, __ldcg(a.part_ml + (base + c) * 2));
+        for (int w = 0; w < wpp; ++w) M = fmaxf(M, sm->att_s[buf][w0i + w][DH]);
         float L = 0.f, A[EPL];
 #pragma unroll
         for (int j = 0; j < EPL; ++j) A[j] = 0.f;
-        for (int c = 0; c < nch; ++c) {
-          const float w = exp2f(__ldcg(a.part_ml + (base + c) * 2) - M);
-          L += __ldcg(a.part_ml + (base + c) * 2 + 1) * w;
+        for (int w = 0; w < wpp; ++w) {
+          const float mw = sm->att_s[buf][w0i + w][DH];
+          const float wt = (mw == -CUDART_INF_F) ? 0.f : exp2f(mw - M);
+          L += sm->att_s[buf][w0i + w][DH + 1] * wt;
 #pragma unroll
-          for (int j = 0; j < EPL; ++j) A[j] += __ldcg(a.part_acc + (base + c) * DH + lane + 32 * j) * w;
+          for (int j = 0; j < EPL; ++j) A[j] += sm->att_s[buf][w0i + w][lane + 32 * j] * wt;
         }
         const float il = 1.f / L;
 #pragma unroll
         for (int j = 0; j < EPL; ++j) a.o[(size_t)r * d + hd * DH + lane + 32 * j] = __float2bfloat16_rn(A[j] * il);
-        if (lane == 0) a.attn_count[r * H + hd] = 0;
       }
+      buf ^= 1;
     }
-    __syncwarp();
   }
 }
 
 // ---- stage: SwiGLU ----------------------------------------------------------------------------------
-__device__ void stage_swiglu(const MegaArgs& a, int wtid) {
+// 8 consecutive features per thread (two 128-bit loads per partial segment, one 128-bit store).
+__device__ void stage_swiglu(const MegaArgs& a, MegaSmem* sm, int wtid) {
   const MegaGemmShape& gs = a.shape[2];
-  const long long n = (long long)a.B * a.F;
+  stage_inv_rms(a, sm, wtid);
+  const int F8 = a.F >> 3;
+  const long long n = (long long)a.B * F8;
   for (long long e = (long long)blockIdx.x * kMegaWorkers + wtid; e < n; e += (long long)gridDim.x * kMegaWorkers) {
-    const int r = (int)(e / a.F), f = (int)(e - (long long)r * a.F);
+    const int r = (int)(e / F8), f0 = (int)(e - (long long)r * F8) << 3;
     if (!a.st.active[r]) continue;
-    const float inv = row_inv_rms(a, r);
-    const float gt = inv * sum_partials_cg(a.partial, gs, a.NT, f, r);
-    const float up = inv * sum_partials_cg(a.partial, gs, a.NT, a.F + f, r);
-    a.act[(size_t)r * a.F + f] = __float2bfloat16_rn(gt / (1.f + __expf(-gt)) * up);
+    const float inv = sm->inv_s[r];
+    float gt[8], up[8];
+    sum_partials8_cg(a.partial, gs, a.NT, f0, r, gt);
+    sum_partials8_cg(a.partial, gs, a.NT, a.F + f0, r, up);
+    __align__(16) bf16 ob[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const float gv = gt[j] * inv;
+      ob[j] = __float2bfloat16_rn(gv / (1.f + __expf(-gv)) * (up[j] * inv));
+    }
+    *reinterpret_cast<uint4*>(a.act + (size_t)r * a.F + f0) = *reinterpret_cast<const uint4*>(ob);
   }
 }
 
@@ -486,20 +483,25 @@ __device__ void stage_tile_argmax(const MegaArgs& a, MegaSmem* sm, int wtid) {
   const int half_id = wtid >> 7, t128 = wtid & 127, lane = wtid & 31, w4 = t128 >> 5;
   uint32_t* s_key = &sm->am_key[half_id][0][0];       // [4 warps][64 batch rows]
   int* s_id = &sm->am_id[half_id][0][0];
+  stage_inv_rms(a, sm, wtid);
+  const size_t slot_stride = (size_t)a.NT * 128, cta_stride = slot_stride * gs.max_seg;
   for (int tile0 = blockIdx.x * 2; tile0 < a.n_tiles_lm; tile0 += gridDim.x * 2) {
     const int tile = tile0 + half_id;
     const bool tile_ok = tile < a.n_tiles_lm;
     const int v = tile * 128 + t128;
+    int4 ts = make_int4(0, 1, 0, 0);
+    if (tile_ok) ts = __ldg(reinterpret_cast<const int4*>(gs.tiles) + tile);
     for (int rb = 0; rb < a.B; rb += 64) {              // 64 batch rows at a time (scratch holds 4 x 64 per half)
       const int rend = min(a.B, rb + 64);
       for (int r = rb; r < rend; ++r) {
         uint32_t key = 0;
-        if (tile_ok && a.st.active[r]) {
-          if (v < a.V) {
-            const float lg = row_inv_rms(a, r) * sum_partials_cg(a.partial, gs, a.NT, v, r);
-            if (a.dump_logits) a.dump_logits[(size_t)r * a.V + v] = lg;
-            if (!(a.st.eos_at[r] > 0 && v == a.eos_id)) key = float_order_key(lg);
-          }
+        if (tile_ok && a.st.active[r] && v < a.V) {
+          const size_t off = (size_t)r * 128 + t128;
+          float lg = __ldcg(a.partial + (size_t)ts.x * slot_stride + off);
+          for (int c = ts.y; c <= ts.z; ++c) lg += __ldcg(a.partial + (size_t)c * cta_stride + off);
+          lg *= sm->inv_s[r];
+          if (a.dump_logits) a.dump_logits[(size_t)r * a.V + v] = lg;
+          if (!(a.st.eos_at[r] > 0 && v == a.eos_id)) key = float_order_key(lg);
         }
         const uint32_t best = __reduce_max_sync(0xffffffffu, key);
         const uint32_t who = __ballot_sync(0xffffffffu, key == best);
@@ -787,7 +789,7 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
       } else if (type == 1) {
         stage_residual(a, sm, wtid, 1, &a.shape[1], a.norm_ptr[2 * layer + 1], false);
       } else if (type == 2) {
-        stage_swiglu(a, wtid);
+        stage_swiglu(a, sm, wtid);
       } else if (type == 3) {
         stage_residual(a, sm, wtid, 1, &a.shape[3], a.norm_ptr[2 * layer + 2], layer + 1 == a.n_layers);
       } else {

@@ -430,6 +430,13 @@ int enqueue_decode_step(ss_ctx* c, const ss_step_opts* opts, int32_t* next_token
   a.st = c->st; a.kv = c->kv;
   a.h = c->h_dec; a.x = c->x_dec; a.o = c->o_dec; a.act = c->act_dec;
   a.rowss = c->rowss; a.partial = c->partial;
+  {
+    // enough (row, head) items for about two rounds over all worker-warp groups
+    const long long pairs = (long long)B * m.n_heads;
+    int wpp = 8;
+    while (wpp > 1 && pairs * wpp > 2LL * c->n_sm * 8) wpp >>= 1;
+    a.attn_wpp = wpp;
+  }
   a.part_ml = c->part_ml; a.part_acc = c->part_acc; a.attn_count = c->attn_count; a.max_chunks = c->max_chunks;
   a.tile_val = c->tile_val; a.tile_idx = c->tile_idx; a.n_tiles_lm = c->n_tiles_lm;
   a.forced = opts ? opts->forced_tokens : nullptr;
