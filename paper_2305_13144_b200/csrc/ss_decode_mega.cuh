@@ -261,7 +261,7 @@ __device__ void stage_attention(const MegaArgs& a, MegaSmem* sm, int wtid, int l
   constexpr int GROUP = DH / 8;            // lanes per key
   constexpr int KPW = 32 / GROUP;          // keys per warp-wide load
   constexpr int HL = GROUP / 2;            // lanes holding the first half of the head
-  constexpr int U = 8;                     // warp-wide loads in flight (K and V each)
+  constexpr int U = 4;                     // warp-wide loads per batch (K and V each); two batches in flight
   constexpr int EPL = DH / 32;
   const int lane = wtid & 31, wid = wtid >> 5;
   const int gl = lane % GROUP, g = lane / GROUP;
@@ -280,6 +280,35 @@ __device__ void stage_attention(const MegaArgs& a, MegaSmem* sm, int wtid, int l
     if (!a.st.active[r]) continue;                   // uniform within the group
     const int pos = a.st.ctx_len[r];                 // new token's position; cached tokens are 0..pos-1
     const float inv = sm->inv_s[r];
+
+    // ---- software-pipelined scan of this warp's pages: the loads of batch b+1 are in flight while
+    // batch b is folded into the running softmax.  A batch is U warp-wide loads = U*KPW tokens.
+    constexpr int BT = KPW * U;                      // tokens per batch
+    constexpr int BPP = kPageTokens / BT;            // batches per page
+    const int npg = (pos + kPageTokens - 1) / kPageTokens;
+    const int my_pages = npg > wig ? (npg - wig + wpp - 1) / wpp : 0;
+    const int n_batches = my_pages * BPP;
+    const int32_t* bt_row = a.st.block_table + (size_t)r * a.st.max_pages;
+    uint4 kk[2][U], vv[2][U];
+    auto issue = [&](int b, uint4 (&kd)[U], uint4 (&vd)[U]) {
+      const int pi = wig + (b / BPP) * wpp;
+      int pg = bt_row[pi];
+      if (pg < 0 || pg >= a.kv.n_pages) { atomicCAS(a.status, 0u, (uint32_t)kStatusBadPage); pg = 0; }
+      const int tcount = min(kPageTokens, pos - pi * kPageTokens);
+      const bf16* kb = kv_layer + (size_t)pg * a.kv.page_elems + (size_t)hd * kPageTokens * DH + gl * 8;
+      const int tb = (b % BPP) * BT;
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const int t = tb + u * KPW + g;
+        kd[u] = make_uint4(0, 0, 0, 0);
+        vd[u] = kd[u];
+        if (t < tcount) {
+          kd[u] = __ldg(reinterpret_cast<const uint4*>(kb + (size_t)t * DH));
+          vd[u] = __ldg(reinterpret_cast<const uint4*>(kb + (size_t)t * DH + v_off));
+        }
+      }
+    };
+    if (n_batches > 0) issue(0, kk[0], vv[0]);
 
     // rotation angles of this lane's 8 dimensions (index within the half)
     float sn[8], cs[8];
@@ -306,56 +335,47 @@ __device__ void stage_attention(const MegaArgs& a, MegaSmem* sm, int wtid, int l
 #pragma unroll
     for (int j = 0; j < 8; ++j) acc[j] = 0.f;
 
-    const int npg = (pos + kPageTokens - 1) / kPageTokens;
-    for (int pi = wig; pi < npg; pi += wpp) {
-      int pg = a.st.block_table[(size_t)r * a.st.max_pages + pi];
-      if (pg < 0 || pg >= a.kv.n_pages) { atomicCAS(a.status, 0u, (uint32_t)kStatusBadPage); pg = 0; }
+    auto fold = [&](int b, const uint4 (&kd)[U], const uint4 (&vd)[U]) {
+      const int pi = wig + (b / BPP) * wpp;
       const int tcount = min(kPageTokens, pos - pi * kPageTokens);
-      const bf16* kb = kv_layer + (size_t)pg * a.kv.page_elems + (size_t)hd * kPageTokens * DH + gl * 8;
-      for (int tb = 0; tb < tcount; tb += KPW * U) {
-        uint4 kk[U], vv[U];
-        bool valid[U];
+      const int tb = (b % BPP) * BT;
+      float s[U];
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-          const int t = tb + u * KPW + g;
-          valid[u] = t < tcount;
-          kk[u] = make_uint4(0, 0, 0, 0);
-          vv[u] = kk[u];
-          if (valid[u]) {
-            kk[u] = __ldg(reinterpret_cast<const uint4*>(kb + (size_t)t * DH));
-            vv[u] = __ldg(reinterpret_cast<const uint4*>(kb + (size_t)t * DH + v_off));
-          }
+      for (int u = 0; u < U; ++u) {
+        float kf[8], dot = 0.f;
+        unpack8(kd[u], kf);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) dot += q[j] * kf[j];
+#pragma unroll
+        for (int o = GROUP / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+        s[u] = (tb + u * KPW + g < tcount) ? dot : -CUDART_INF_F;
+      }
+      float mn = m;
+#pragma unroll
+      for (int u = 0; u < U; ++u) mn = fmaxf(mn, s[u]);
+      const float sc = (mn == -CUDART_INF_F) ? 1.f : exp2f(m - mn);
+      l *= sc;
+#pragma unroll
+      for (int j = 0; j < 8; ++j) acc[j] *= sc;
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        if (s[u] != -CUDART_INF_F) {
+          const float pw = exp2f(s[u] - mn);
+          float vf[8];
+          unpack8(vd[u], vf);
+          l += pw;
+#pragma unroll
+          for (int j = 0; j < 8; ++j) acc[j] += pw * vf[j];
         }
-        float s[U];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-          float kf[8], dot = 0.f;
-          unpack8(kk[u], kf);
-#pragma unroll
-          for (int j = 0; j < 8; ++j) dot += q[j] * kf[j];
-#pragma unroll
-          for (int o = GROUP / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-          s[u] = valid[u] ? dot : -CUDART_INF_F;
-        }
-        float mn = m;
-#pragma unroll
-        for (int u = 0; u < U; ++u) mn = fmaxf(mn, s[u]);
-        const float sc = (mn == -CUDART_INF_F) ? 1.f : exp2f(m - mn);
-        l *= sc;
-#pragma unroll
-        for (int j = 0; j < 8; ++j) acc[j] *= sc;
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-          if (valid[u]) {
-            const float pw = exp2f(s[u] - mn);
-            float vf[8];
-            unpack8(vv[u], vf);
-            l += pw;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) acc[j] += pw * vf[j];
-          }
-        }
-        m = mn;
+      }
+      m = mn;
+    };
+    for (int b = 0; b < n_batches; b += 2) {
+      if (b + 1 < n_batches) issue(b + 1, kk[1], vv[1]);
+      fold(b, kk[0], vv[0]);
+      if (b + 1 < n_batches) {
+        if (b + 2 < n_batches) issue(b + 2, kk[0], vv[0]);
+        fold(b + 1, kk[1], vv[1]);
       }
     }
 
