@@ -106,7 +106,9 @@ struct MegaSmem {
   volatile int abort;
   int prefix[kMaxBatch + 1];
   float inv_s[kMaxBatch];          // 1/rms of every row for the running stage
-  float att_s[2][8][136];          // attention: per worker warp (acc[Dh], max, sum), double-buffered
+  __align__(16) float q_s[8][128]; // attention: per worker warp, rotated query (then the new token's value); read as float4
+  __align__(16) float att_s[8][9][132];   // attention: [pair of the pass][partial: 8 warps + new token][acc[Dh], max, sum]
+  int pair_id[8], pair_ustart[9], pair_n, pair_next, pair_lo, pair_hi;
   float red[8];
   uint32_t am_key[2][4][64];       // per-tile arg-max scratch: [tile half][warp][batch row]
   int am_id[2][4][64];
@@ -132,6 +134,7 @@ __device__ __forceinline__ bool mega_wait(uint32_t bar, uint32_t parity, MegaSme
       sm->abort = 1;
       return false;
     }
+    __nanosleep(40);                 // a spinning role must not starve the warps that share its scheduler
   }
 }
 
@@ -250,225 +253,329 @@ __device__ __forceinline__ void group_bar(int id, int threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
+// ---- ahead of the attention stage: pull the cached keys/values it will read into L2 -------------------------
+// Called by the workers while the qkv projection streams its weights (they would otherwise only wait
+// for the accumulators).  Same (row, head) -> warp -> page mapping as stage_attention, one 128-byte
+// line per prefetch, no registers held and nothing to wait for.
+template <int DH>
+__device__ void attention_prefetch(const MegaArgs& a, int wtid, int layer) {
+  const int lane = wtid & 31, wid = wtid >> 5;
+  const int wpp = a.attn_wpp, grp = wid / wpp, wig = wid - grp * wpp, GP = 8 / wpp;
+  const int H = a.H;
+  const uint8_t* kv_layer = reinterpret_cast<const uint8_t*>(a.kv.pool + (size_t)layer * a.kv.layer_stride);
+  const size_t v_off = (size_t)H * kPageTokens * DH * 2;
+  const int n_pairs = a.B * H;
+  for (int p = blockIdx.x * GP + grp; p < n_pairs; p += gridDim.x * GP) {
+    const int r = p / H, hd = p - r * H;
+    if (!a.st.active[r]) continue;
+    const int pos = a.st.ctx_len[r];
+    const int npg = (pos + kPageTokens - 1) / kPageTokens;
+    for (int pi = wig; pi < npg; pi += wpp) {
+      const int pg = a.st.block_table[(size_t)r * a.st.max_pages + pi];
+      if (pg < 0 || pg >= a.kv.n_pages) continue;
+      const int bytes = min(kPageTokens, pos - pi * kPageTokens) * DH * 2;
+      const uint8_t* kb = kv_layer + ((size_t)pg * a.kv.page_elems + (size_t)hd * kPageTokens * DH) * 2;
+      for (int off = lane * 128; off < bytes; off += 32 * 128) {
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(kb + off));
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(kb + v_off + off));
+      }
+    }
+  }
+}
+
 // ---- stage: q,k,v from partials + RoPE + cache append + paged attention ----------------------------------
-// Work item = (row, head).  A group of `wpp` warps of one CTA shares an item: every warp rebuilds the
-// rotated query (cheap, and it avoids a hand-off), takes every wpp-th page of the row's cache, and
-// leaves its running (max, sum, acc) in shared memory; the group's first warp also builds k,v of
-// the new token, appends them to the page, attends to them from registers and merges the group.
-// A lane owns 8 consecutive head dimensions (one 128-bit load); Dh/8 lanes cover a key.
+// Work is dealt in units of (row, head, page of 32 cached tokens).  Every CTA owns a contiguous run of
+// (row, head) pairs holding about 1/gridDim of all units (pairs are not split across CTAs, so their
+// partial results meet in shared memory).  A CTA works through its pairs in passes of up to 8:
+//   A  warp j builds pair j's rotated query (shared memory) and the new token's k,v: appended to the
+//      page, and entered as the pair's ninth partial (score, 1, v);
+//   B  the pass's units are cut into 8 equal contiguous slices, one per warp; a warp scans its pages
+//      and leaves one (max, sum, acc) partial per pair it touched;
+//   C  warp j merges pair j's partials and writes the bf16 output.
+// Scan layout: a key row is Dh/8 chunks of 16 bytes; lane (g, gl) of the warp handles key g of the
+// load step and chunks gl, gl+GROUP, gl+2*GROUP, gl+3*GROUP, so each warp-wide load reads 64
+// contiguous bytes per key (full sectors).
+template <int N>
+__device__ __forceinline__ void sum_partialsN_cg(const float* __restrict__ partial, const MegaGemmShape& s, int NT, int n0,
+                                                 int tok, float (&x)[N]) {
+  static_assert(N == 2 || N == 4, "N");
+  const int4 t = __ldg(reinterpret_cast<const int4*>(s.tiles) + (n0 >> 7));
+  const size_t slot_stride = (size_t)NT * 128, cta_stride = slot_stride * s.max_seg;
+  const size_t off = (size_t)tok * 128 + (n0 & 127);
+  auto add = [&](const float* p, bool first) {
+    if constexpr (N == 4) {
+      const float4 u = __ldcg(reinterpret_cast<const float4*>(p));
+      if (first) { x[0] = u.x; x[1] = u.y; x[2] = u.z; x[3] = u.w; }
+      else { x[0] += u.x; x[1] += u.y; x[2] += u.z; x[3] += u.w; }
+    } else {
+      const float2 u = __ldcg(reinterpret_cast<const float2*>(p));
+      if (first) { x[0] = u.x; x[1] = u.y; }
+      else { x[0] += u.x; x[1] += u.y; }
+    }
+  };
+  add(partial + (size_t)t.x * slot_stride + off, true);
+  for (int c = t.y; c <= t.z; ++c) add(partial + (size_t)c * cta_stride + off, false);
+}
+
+constexpr int kAttnPass = 8;               // pairs per pass (= worker warps)
+constexpr int kAttnSlots = 9;              // partials per pair: one per warp + the new token
+
 template <int DH>
 __device__ void stage_attention(const MegaArgs& a, MegaSmem* sm, int wtid, int layer) {
-  constexpr int GROUP = DH / 8;            // lanes per key
-  constexpr int KPW = 32 / GROUP;          // keys per warp-wide load
-  constexpr int HL = GROUP / 2;            // lanes holding the first half of the head
-  constexpr int U = 4;                     // warp-wide loads per batch (K and V each); two batches in flight
-  constexpr int EPL = DH / 32;
+  constexpr int GROUP = DH / 32;           // lanes per key in the cache scan
+  constexpr int KPW = 32 / GROUP;          // keys per warp-wide load step
+  constexpr int EPL = DH / 32;             // cooperative layout: consecutive dimensions per lane
+  constexpr int STEPS = kPageTokens / KPW; // load steps per page (4 at Dh 128, 2 at Dh 64)
+  constexpr int U = 2;                     // load steps per batch
   const int lane = wtid & 31, wid = wtid >> 5;
   const int gl = lane % GROUP, g = lane / GROUP;
-  const int wpp = a.attn_wpp, grp = wid / wpp, wig = wid - grp * wpp, GP = 8 / wpp;
-  const int H = a.H, d = a.d;
+  const int H = a.H, d = a.d, B = a.B;
   const MegaGemmShape& gs = a.shape[0];
   const float qscale = rsqrtf((float)DH) * 1.4426950408889634f;
   const bf16* kv_layer = a.kv.pool + (size_t)layer * a.kv.layer_stride;
   const size_t v_off = (size_t)H * kPageTokens * DH;
-  const int n_pairs = a.B * H;
-  stage_inv_rms(a, sm, wtid);
-  int buf = 0;
 
-  for (int p = blockIdx.x * GP + grp; p < n_pairs; p += gridDim.x * GP) {
-    const int r = p / H, hd = p - r * H;
-    if (!a.st.active[r]) continue;                   // uniform within the group
-    const int pos = a.st.ctx_len[r];                 // new token's position; cached tokens are 0..pos-1
-    const float inv = sm->inv_s[r];
-
-    // ---- software-pipelined scan of this warp's pages: the loads of batch b+1 are in flight while
-    // batch b is folded into the running softmax.  A batch is U warp-wide loads = U*KPW tokens.
-    constexpr int BT = KPW * U;                      // tokens per batch
-    constexpr int BPP = kPageTokens / BT;            // batches per page
-    const int npg = (pos + kPageTokens - 1) / kPageTokens;
-    const int my_pages = npg > wig ? (npg - wig + wpp - 1) / wpp : 0;
-    const int n_batches = my_pages * BPP;
-    const int32_t* bt_row = a.st.block_table + (size_t)r * a.st.max_pages;
-    uint4 kk[2][U], vv[2][U];
-    auto issue = [&](int b, uint4 (&kd)[U], uint4 (&vd)[U]) {
-      const int pi = wig + (b / BPP) * wpp;
-      int pg = bt_row[pi];
-      if (pg < 0 || pg >= a.kv.n_pages) { atomicCAS(a.status, 0u, (uint32_t)kStatusBadPage); pg = 0; }
-      const int tcount = min(kPageTokens, pos - pi * kPageTokens);
-      const bf16* kb = kv_layer + (size_t)pg * a.kv.page_elems + (size_t)hd * kPageTokens * DH + gl * 8;
-      const int tb = (b % BPP) * BT;
+  // ---- pages per row (exclusive prefix, active rows only) and this CTA's run of pairs
+  if (wid == 0) {
+    int cnt[8], loc = 0;
 #pragma unroll
-      for (int u = 0; u < U; ++u) {
-        const int t = tb + u * KPW + g;
-        kd[u] = make_uint4(0, 0, 0, 0);
-        vd[u] = kd[u];
-        if (t < tcount) {
-          kd[u] = __ldg(reinterpret_cast<const uint4*>(kb + (size_t)t * DH));
-          vd[u] = __ldg(reinterpret_cast<const uint4*>(kb + (size_t)t * DH + v_off));
-        }
-      }
-    };
-    if (n_batches > 0) issue(0, kk[0], vv[0]);
-
-    // rotation angles of this lane's 8 dimensions (index within the half)
-    float sn[8], cs[8];
-    {
-      const int f0 = (gl % HL) * 8;
-#pragma unroll
-      for (int j = 0; j < 8; ++j) sincosf((float)pos * a.inv_freq[f0 + j], &sn[j], &cs[j]);
+    for (int j = 0; j < 8; ++j) {
+      const int r = lane * 8 + j;
+      int c = 0;
+      if (r < B && a.st.active[r]) c = (a.st.ctx_len[r] + kPageTokens - 1) / kPageTokens;
+      cnt[j] = c;
+      loc += c;
     }
-    // q: partial sums, lazy norm, RoPE (partner dimension lives HL lanes away), bf16 rounding
-    float q[8];
-    {
-      float x[8];
-      sum_partials8_cg(a.partial, gs, a.NT, hd * DH + gl * 8, r, x);
+    int inc = loc;
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const float xv = x[j] * inv;
-        const float pv = __shfl_xor_sync(0xffffffffu, xv, HL);
-        const float o = (gl < HL) ? xv * cs[j] - pv * sn[j] : xv * cs[j] + pv * sn[j];
-        q[j] = __bfloat162float(__float2bfloat16_rn(o)) * qscale;
-      }
+    for (int o = 1; o < 32; o <<= 1) {
+      const int t = __shfl_up_sync(0xffffffffu, inc, o);
+      if (lane >= o) inc += t;
     }
-
-    float m = -CUDART_INF_F, l = 0.f, acc[8];
+    int run = inc - loc;
 #pragma unroll
-    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
-
-    auto fold = [&](int b, const uint4 (&kd)[U], const uint4 (&vd)[U]) {
-      const int pi = wig + (b / BPP) * wpp;
-      const int tcount = min(kPageTokens, pos - pi * kPageTokens);
-      const int tb = (b % BPP) * BT;
-      float s[U];
-#pragma unroll
-      for (int u = 0; u < U; ++u) {
-        float kf[8], dot = 0.f;
-        unpack8(kd[u], kf);
-#pragma unroll
-        for (int j = 0; j < 8; ++j) dot += q[j] * kf[j];
-#pragma unroll
-        for (int o = GROUP / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-        s[u] = (tb + u * KPW + g < tcount) ? dot : -CUDART_INF_F;
-      }
-      float mn = m;
-#pragma unroll
-      for (int u = 0; u < U; ++u) mn = fmaxf(mn, s[u]);
-      const float sc = (mn == -CUDART_INF_F) ? 1.f : exp2f(m - mn);
-      l *= sc;
-#pragma unroll
-      for (int j = 0; j < 8; ++j) acc[j] *= sc;
-#pragma unroll
-      for (int u = 0; u < U; ++u) {
-        if (s[u] != -CUDART_INF_F) {
-          const float pw = exp2f(s[u] - mn);
-          float vf[8];
-          unpack8(vd[u], vf);
-          l += pw;
-#pragma unroll
-          for (int j = 0; j < 8; ++j) acc[j] += pw * vf[j];
-        }
-      }
-      m = mn;
-    };
-    for (int b = 0; b < n_batches; b += 2) {
-      if (b + 1 < n_batches) issue(b + 1, kk[1], vv[1]);
-      fold(b, kk[0], vv[0]);
-      if (b + 1 < n_batches) {
-        if (b + 2 < n_batches) issue(b + 2, kk[0], vv[0]);
-        fold(b + 1, kk[1], vv[1]);
-      }
+    for (int j = 0; j < 8; ++j) {
+      sm->prefix[lane * 8 + j] = run;
+      run += cnt[j];
     }
+    if (lane == 31) sm->prefix[kMaxBatch] = inc;
+    if (lane == 0) { sm->pair_lo = 0x7fffffff; sm->pair_hi = -1; }
+  }
+  named_bar_workers();
+  {
+    const long long T = (long long)sm->prefix[kMaxBatch] * H;        // all units
+    const long long lo = (long long)blockIdx.x * T / gridDim.x, hi = (long long)(blockIdx.x + 1) * T / gridDim.x;
+    int mylo = 0x7fffffff, myhi = -1;
+    for (int p = wtid; p < B * H; p += kMegaWorkers) {
+      const int r = p / H, hd = p - r * H;
+      const int npr = sm->prefix[r + 1] - sm->prefix[r];     // pages of this row (0 if inactive)
+      if (npr <= 0) continue;
+      const long long cum = (long long)sm->prefix[r] * H + (long long)hd * npr;   // units before this pair
+      if (cum >= lo && cum < hi) { mylo = min(mylo, p); myhi = max(myhi, p); }
+    }
+    if (mylo <= myhi) { atomicMin(&sm->pair_lo, mylo); atomicMax(&sm->pair_hi, myhi); }
+  }
+  named_bar_workers();
+  const int p_begin = sm->pair_lo, p_end = sm->pair_hi + 1;          // empty run: lo > hi
 
-    if (wig == 0) {
-      // the new token: k (rotated), v -> bf16 -> page; its score and value straight from registers
-      float kx[8], vx[8];
-      sum_partials8_cg(a.partial, gs, a.NT, d + hd * DH + gl * 8, r, kx);
-      sum_partials8_cg(a.partial, gs, a.NT, 2 * d + hd * DH + gl * 8, r, vx);
-      __align__(16) bf16 kb8[8], vb8[8];
-      float dot = 0.f;
-#pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const float xv = kx[j] * inv;
-        const float pv = __shfl_xor_sync(0xffffffffu, xv, HL);
-        const float o = (gl < HL) ? xv * cs[j] - pv * sn[j] : xv * cs[j] + pv * sn[j];
-        kb8[j] = __float2bfloat16_rn(o);
-        vb8[j] = __float2bfloat16_rn(vx[j] * inv);
-        dot += q[j] * __bfloat162float(kb8[j]);
+  for (int pass0 = p_begin; pass0 < p_end; ) {
+    // ---- the pass: next (up to 8) pairs with work; pair_id / pair_pages / pair_ustart in shared memory
+    if (wid == 0) {
+      int n = 0, p = pass0, ustart = 0;
+      // lanes walk the pairs together (few iterations: rows without work are skipped by whole rows)
+      while (p < p_end && n < kAttnPass) {
+        const int r = p / H;
+        const int npr = sm->prefix[r + 1] - sm->prefix[r];
+        if (npr <= 0) { p = (r + 1) * H; continue; }
+        if (lane == 0) { sm->pair_id[n] = p; sm->pair_ustart[n] = ustart; }
+        ustart += npr;
+        ++n;
+        ++p;
       }
+      if (lane == 0) { sm->pair_n = n; sm->pair_next = p; sm->pair_ustart[n] = ustart; }
+    }
+    for (int i = wtid; i < kAttnPass * kAttnSlots; i += kMegaWorkers) sm->att_s[i / kAttnSlots][i % kAttnSlots][DH] = -CUDART_INF_F;
+    named_bar_workers();
+    const int np_pass = sm->pair_n;
+    const int U_pass = sm->pair_ustart[np_pass];
+
+    // ---- A: warp j prepares pair j
+    if (wid < np_pass) {
+      const int p = sm->pair_id[wid];
+      const int r = p / H, hd = p - r * H;
+      const int pos = a.st.ctx_len[r];
+      const float inv = row_inv_rms(a, r);
+      const int e0 = lane * EPL;
+      float sn[EPL], cs[EPL];
 #pragma unroll
-      for (int o = GROUP / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+      for (int j = 0; j < EPL; ++j) sincosf((float)pos * a.inv_freq[(lane & 15) * EPL + j], &sn[j], &cs[j]);
+      float qx[EPL], kx[EPL], vx[EPL];
+      sum_partialsN_cg<EPL>(a.partial, gs, a.NT, hd * DH + e0, r, qx);
+      sum_partialsN_cg<EPL>(a.partial, gs, a.NT, d + hd * DH + e0, r, kx);
+      sum_partialsN_cg<EPL>(a.partial, gs, a.NT, 2 * d + hd * DH + e0, r, vx);
       int pg = a.st.block_table[(size_t)r * a.st.max_pages + pos / kPageTokens];
       if (pg < 0 || pg >= a.kv.n_pages) { atomicCAS(a.status, 0u, (uint32_t)kStatusBadPage); pg = -1; }
-      if (g == 0) {
-        if (pg >= 0) {
-          bf16* kdst = a.kv.pool + (size_t)layer * a.kv.layer_stride + (size_t)pg * a.kv.page_elems +
-                       ((size_t)hd * kPageTokens + (pos % kPageTokens)) * DH + gl * 8;
-          *reinterpret_cast<uint4*>(kdst) = *reinterpret_cast<const uint4*>(kb8);
-          *reinterpret_cast<uint4*>(kdst + v_off) = *reinterpret_cast<const uint4*>(vb8);
-        }
-        const float mn = fmaxf(m, dot);
-        const float sc = (m == -CUDART_INF_F) ? 0.f : exp2f(m - mn);
-        const float pw = exp2f(dot - mn);
-        l = l * sc + pw;
+      bf16* kdst = a.kv.pool + (size_t)layer * a.kv.layer_stride + (size_t)(pg < 0 ? 0 : pg) * a.kv.page_elems +
+                   ((size_t)hd * kPageTokens + (pos % kPageTokens)) * DH + e0;
+      float dot = 0.f;
+      float* qs = sm->q_s[wid];
+      float* ns = sm->att_s[wid][kAttnSlots - 1];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) acc[j] = acc[j] * sc + pw * __bfloat162float(vb8[j]);
-        m = mn;
+      for (int j = 0; j < EPL; ++j) {
+        const float xq = qx[j] * inv, xk = kx[j] * inv;
+        const float pq = __shfl_xor_sync(0xffffffffu, xq, 16), pk = __shfl_xor_sync(0xffffffffu, xk, 16);
+        const float oq = (lane < 16) ? xq * cs[j] - pq * sn[j] : xq * cs[j] + pq * sn[j];
+        const float ok = (lane < 16) ? xk * cs[j] - pk * sn[j] : xk * cs[j] + pk * sn[j];
+        const float qf = __bfloat162float(__float2bfloat16_rn(oq)) * qscale;
+        const bf16 kb16 = __float2bfloat16_rn(ok), vb16 = __float2bfloat16_rn(vx[j] * inv);
+        if (pg >= 0) { kdst[j] = kb16; kdst[v_off + j] = vb16; }
+        qs[e0 + j] = qf;
+        ns[e0 + j] = __bfloat162float(vb16);
+        dot += qf * __bfloat162float(kb16);
       }
+      dot = warp_sum(dot);
+      if (lane == 0) { ns[DH] = dot; ns[DH + 1] = 1.f; }
     }
+    named_bar_workers();
 
-    // merge the KPW key groups of the warp (same gl, different g)
+    // ---- B: this warp's slice of the pass's units
+    {
+      const int u0 = (int)((long long)wid * U_pass / 8), u1 = (int)((long long)(wid + 1) * U_pass / 8);
+      int j = 0;
+      while (j + 1 < np_pass && sm->pair_ustart[j + 1] <= u0) ++j;
+      float m = -CUDART_INF_F, l = 0.f, acc[32];
 #pragma unroll
-    for (int o = GROUP; o < 32; o <<= 1) {
-      const float om = __shfl_xor_sync(0xffffffffu, m, o);
-      const float ol = __shfl_xor_sync(0xffffffffu, l, o);
-      const float mn = fmaxf(m, om);
-      const float w0 = (m == -CUDART_INF_F) ? 0.f : exp2f(m - mn);
-      const float w1 = (om == -CUDART_INF_F) ? 0.f : exp2f(om - mn);
-      l = l * w0 + ol * w1;
+      for (int e = 0; e < 32; ++e) acc[e] = 0.f;
+      auto flush = [&](int jj) {
+        // merge the KPW key slots of the warp, then lanes of key slot 0 store the partial
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const float oa = __shfl_xor_sync(0xffffffffu, acc[j], o);
-        acc[j] = acc[j] * w0 + oa * w1;
-      }
-      m = mn;
-    }
-
-    if (wpp == 1) {
-      if (g == 0) {
-        const float il = 1.f / l;
-        __align__(16) bf16 ob[8];
+        for (int o = GROUP; o < 32; o <<= 1) {
+          const float om = __shfl_xor_sync(0xffffffffu, m, o);
+          const float ol = __shfl_xor_sync(0xffffffffu, l, o);
+          const float mn = fmaxf(m, om);
+          const float w0 = (m == -CUDART_INF_F) ? 0.f : exp2f(m - mn);
+          const float w1 = (om == -CUDART_INF_F) ? 0.f : exp2f(om - mn);
+          l = l * w0 + ol * w1;
 #pragma unroll
-        for (int j = 0; j < 8; ++j) ob[j] = __float2bfloat16_rn(acc[j] * il);
-        *reinterpret_cast<uint4*>(a.o + (size_t)r * d + hd * DH + gl * 8) = *reinterpret_cast<const uint4*>(ob);
-      }
-    } else {
-      float* slot = sm->att_s[buf][wid];
-      if (g == 0) {
-#pragma unroll
-        for (int j = 0; j < 8; ++j) slot[gl * 8 + j] = acc[j];
-        if (gl == 0) { slot[DH] = m; slot[DH + 1] = l; }
-      }
-      group_bar(2 + grp, wpp * 32);
-      if (wig == 0) {
-        const int w0i = grp * wpp;
-        float M = -CUDART_INF_F;
-        for (int w = 0; w < wpp; ++w) M = fmaxf(M, sm->att_s[buf][w0i + w][DH]);
-        float L = 0.f, A[EPL];
-#pragma unroll
-        for (int j = 0; j < EPL; ++j) A[j] = 0.f;
-        for (int w = 0; w < wpp; ++w) {
-          const float mw = sm->att_s[buf][w0i + w][DH];
-          const float wt = (mw == -CUDART_INF_F) ? 0.f : exp2f(mw - M);
-          L += sm->att_s[buf][w0i + w][DH + 1] * wt;
-#pragma unroll
-          for (int j = 0; j < EPL; ++j) A[j] += sm->att_s[buf][w0i + w][lane + 32 * j] * wt;
+          for (int e = 0; e < 32; ++e) {
+            const float oa = __shfl_xor_sync(0xffffffffu, acc[e], o);
+            acc[e] = acc[e] * w0 + oa * w1;
+          }
+          m = mn;
         }
-        const float il = 1.f / L;
+        float* slot = sm->att_s[jj][wid];
+        if (g == 0) {
 #pragma unroll
-        for (int j = 0; j < EPL; ++j) a.o[(size_t)r * d + hd * DH + lane + 32 * j] = __float2bfloat16_rn(A[j] * il);
+          for (int c = 0; c < 4; ++c)
+#pragma unroll
+            for (int e = 0; e < 8; ++e) slot[(c * GROUP + gl) * 8 + e] = acc[c * 8 + e];
+          if (gl == 0) { slot[DH] = m; slot[DH + 1] = l; }
+        }
+        m = -CUDART_INF_F;
+        l = 0.f;
+#pragma unroll
+        for (int e = 0; e < 32; ++e) acc[e] = 0.f;
+      };
+      for (int u = u0; u < u1; ++u) {
+        if (u >= sm->pair_ustart[j + 1]) { flush(j); ++j; }
+        const int p = sm->pair_id[j];
+        const int r = p / H, hd = p - r * H;
+        const int pi = u - sm->pair_ustart[j];
+        const int pos = a.st.ctx_len[r];
+        int pg = a.st.block_table[(size_t)r * a.st.max_pages + pi];
+        if (pg < 0 || pg >= a.kv.n_pages) { atomicCAS(a.status, 0u, (uint32_t)kStatusBadPage); pg = 0; }
+        const int tcount = min(kPageTokens, pos - pi * kPageTokens);
+        const bf16* kb = kv_layer + (size_t)pg * a.kv.page_elems + (size_t)hd * kPageTokens * DH;
+        const float* qs = sm->q_s[j];
+#pragma unroll 1
+        for (int s0 = 0; s0 < STEPS; s0 += U) {
+          uint4 kk[U][4], vv[U][4];
+#pragma unroll
+          for (int uu = 0; uu < U; ++uu) {
+            const int t = (s0 + uu) * KPW + g;
+            if (t < tcount) {
+              const uint4* kp = reinterpret_cast<const uint4*>(kb + (size_t)t * DH);
+              const uint4* vp = reinterpret_cast<const uint4*>(kb + (size_t)t * DH + v_off);
+#pragma unroll
+              for (int c = 0; c < 4; ++c) { kk[uu][c] = __ldg(kp + c * GROUP + gl); vv[uu][c] = __ldg(vp + c * GROUP + gl); }
+            } else {
+#pragma unroll
+              for (int c = 0; c < 4; ++c) { kk[uu][c] = make_uint4(0, 0, 0, 0); vv[uu][c] = kk[uu][c]; }
+            }
+          }
+          float sc_[U];
+#pragma unroll
+          for (int uu = 0; uu < U; ++uu) {
+            float dot = 0.f;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              float kf[8];
+              unpack8(kk[uu][c], kf);
+              const float4 qa = *reinterpret_cast<const float4*>(qs + (c * GROUP + gl) * 8);
+              const float4 qb = *reinterpret_cast<const float4*>(qs + (c * GROUP + gl) * 8 + 4);
+              dot += qa.x * kf[0] + qa.y * kf[1] + qa.z * kf[2] + qa.w * kf[3] + qb.x * kf[4] + qb.y * kf[5] +
+                     qb.z * kf[6] + qb.w * kf[7];
+            }
+#pragma unroll
+            for (int o = GROUP / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+            sc_[uu] = ((s0 + uu) * KPW + g < tcount) ? dot : -CUDART_INF_F;
+          }
+          float mn = m;
+#pragma unroll
+          for (int uu = 0; uu < U; ++uu) mn = fmaxf(mn, sc_[uu]);
+          if (mn != -CUDART_INF_F) {
+            if (mn != m) {
+              const float sc = exp2f(m - mn);
+              l *= sc;
+#pragma unroll
+              for (int e = 0; e < 32; ++e) acc[e] *= sc;
+              m = mn;
+            }
+#pragma unroll
+            for (int uu = 0; uu < U; ++uu) {
+              if (sc_[uu] != -CUDART_INF_F) {
+                const float pw = exp2f(sc_[uu] - mn);
+                l += pw;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                  float vf[8];
+                  unpack8(vv[uu][c], vf);
+#pragma unroll
+                  for (int e = 0; e < 8; ++e) acc[c * 8 + e] += pw * vf[e];
+                }
+              }
+            }
+          }
+        }
       }
-      buf ^= 1;
+      if (u1 > u0) flush(j);
     }
+    named_bar_workers();
+
+    // ---- C: warp j merges pair j
+    if (wid < np_pass) {
+      const int p = sm->pair_id[wid];
+      const int r = p / H, hd = p - r * H;
+      const int e0 = lane * EPL;
+      float M = -CUDART_INF_F;
+      for (int k = 0; k < kAttnSlots; ++k) M = fmaxf(M, sm->att_s[wid][k][DH]);
+      float L = 0.f, A[EPL];
+#pragma unroll
+      for (int j = 0; j < EPL; ++j) A[j] = 0.f;
+      for (int k = 0; k < kAttnSlots; ++k) {
+        const float mk = sm->att_s[wid][k][DH];
+        if (mk == -CUDART_INF_F) continue;
+        const float wt = exp2f(mk - M);
+        L += sm->att_s[wid][k][DH + 1] * wt;
+#pragma unroll
+        for (int j = 0; j < EPL; ++j) A[j] += sm->att_s[wid][k][e0 + j] * wt;
+      }
+      const float il = 1.f / L;
+#pragma unroll
+      for (int j = 0; j < EPL; ++j) a.o[(size_t)r * d + hd * DH + e0 + j] = __float2bfloat16_rn(A[j] * il);
+    }
+    pass0 = sm->pair_next;
+    named_bar_workers();
   }
 }
 
@@ -591,7 +698,7 @@ template <int DH>
 __global__ void __launch_bounds__(kMegaThreads, 1)
 decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_o,
                         const __grid_constant__ CUtensorMap map_act, const __grid_constant__ MegaArgs a) {
-  extern __shared__ uint8_t smem_raw[];
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
   MegaSmem* sm = reinterpret_cast<MegaSmem*>(smem_raw);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int cta = blockIdx.x, G = gridDim.x;
@@ -672,6 +779,7 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
         {
           const long long t0 = clock64();
           while (sm->act_epoch <= gm) {
+            __nanosleep(100);
             if (sm->abort) { ok = false; break; }
             if (clock64() - t0 > 4000000000LL) {
               atomicCAS(a.status, 0u, (uint32_t)kStatusFlagTimeout);
@@ -687,6 +795,7 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
         for (long long it = it0; it < it1; ++it, ++gi) {
           const long long t0 = clock64();
           while (sm->w_issued <= gi) {
+            __nanosleep(40);
             if (sm->abort) { ok = false; break; }
             if (clock64() - t0 > 4000000000LL) {
               atomicCAS(a.status, 0u, (uint32_t)kStatusFlagTimeout);

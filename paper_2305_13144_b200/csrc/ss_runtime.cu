@@ -431,10 +431,10 @@ int enqueue_decode_step(ss_ctx* c, const ss_step_opts* opts, int32_t* next_token
   a.h = c->h_dec; a.x = c->x_dec; a.o = c->o_dec; a.act = c->act_dec;
   a.rowss = c->rowss; a.partial = c->partial;
   {
-    // enough (row, head) items for about two rounds over all worker-warp groups
+    // one round over the worker-warp groups when the items allow it (the per-item set-up is latency-bound)
     const long long pairs = (long long)B * m.n_heads;
     int wpp = 8;
-    while (wpp > 1 && pairs * wpp > 2LL * c->n_sm * 8) wpp >>= 1;
+    while (wpp > 1 && pairs * wpp > 1LL * c->n_sm * 8) wpp >>= 1;
     a.attn_wpp = wpp;
   }
   a.part_ml = c->part_ml; a.part_acc = c->part_acc; a.attn_count = c->attn_count; a.max_chunks = c->max_chunks;
