@@ -218,3 +218,117 @@ def test_errors_before_launch():
     assert e.value.code == api.SS_ERR_ARG
     api.ss_prefill(eng, toks, [0, 20], None, 4)      # still usable afterwards
     api.ss_release_batch(eng)
+
+
+@pytest.mark.parametrize("B", [40, 130])
+def test_wide_batches_span_several_token_tiles(B):
+    """Batches wider than 16/64 rows: token tiles of 48 and 144 columns, the per-tile arg-max in
+    groups of 64 rows, attention passes of more than 8 (row, head) pairs per CTA."""
+    shape = synth.TINY.with_layers(1)
+    w = synth.make_weights(shape, seed=21)
+    rng = np.random.default_rng(B)
+    lens = rng.integers(3, 70, size=B)
+    prompts = [rng.integers(3, shape.vocab, size=int(n)).tolist() for n in lens]
+    targets = [int(x) for x in rng.integers(1, 4, size=B)]
+    el, eh = _teacher_forced(shape, w, prompts, targets, cap=3, max_batch=256, max_ctx=128, max_prefill=8192,
+                             max_new=8, kv_tokens=256 * 96)
+    assert el <= LOGIT_TOL and eh <= HIDDEN_TOL, (B, el, eh)
+
+
+def test_7b_shape_two_layers_sampled_rows():
+    """The 7B shape (d 4096, 32 heads x 128, FFN 11008, vocab 32000) cut to two layers, batch 16 with the
+    benchmark's prompt lengths; the oracle follows the three rows with the shortest prompts through the
+    prompt pass and two decode steps; all rows run free, and a row is compared for as long as its tokens
+    agree with the oracle's (a disagreement is only accepted on a near-tie of the oracle's top two logits)."""
+    import torch
+    from paper_2305_13144_b200 import api
+    shape = synth.LLAMA_7B.with_layers(2)
+    w = synth.make_weights(shape, seed=7)
+    g = synth.group_7b_batch16(seed=0)
+    B = g.n
+    rows = np.argsort(g.prompt_len)[:3].tolist()
+    model = od.Decoder(w, n_layers=2, n_heads=shape.n_heads, head_dim=shape.head_dim, rms_eps=shape.rms_eps,
+                       rope_theta=shape.rope_theta, eos_id=shape.eos_id, dtype=np.float64)
+    steps = 3
+    ref = {r: od.generate(model, g.prompt(r).tolist(), steps, steps + 5, keep_logits=True, keep_hidden=True) for r in rows}
+    del model
+    eng = api.make_engine(shape, api.runtime_cfg(16, 768, 4096, 512, 16 * 768),
+                          {k: synth.to_bf16_bits(v) for k, v in w.items()})
+    cu = np.zeros(B + 1, dtype=np.int32)
+    cu[1:] = np.cumsum(g.prompt_len)
+    dl = torch.zeros(B, shape.vocab, dtype=torch.float32, device="cuda")
+    dh = torch.zeros(B, shape.d_model, dtype=torch.float32, device="cuda")
+    nxt = torch.zeros(B, dtype=torch.int32, device="cuda")
+    worst_l = worst_h = 0.0
+    for t in range(steps):
+        if t == 0:
+            api.ss_prefill(eng, g.prompt_tokens, cu, np.full(B, steps + 5, dtype=np.int32), 512,
+                           dump_logits=dl, dump_hidden=dh, first_tokens=nxt)
+        else:
+            api.ss_decode_step(eng, dump_logits=dl, dump_hidden=dh, next_tokens=nxt)
+        torch.cuda.synchronize()
+        assert api.ss_last_device_status(eng) == 0
+        gl, gh, gn = dl.cpu().numpy(), dh.cpu().numpy(), nxt.cpu().numpy()
+        for r in rows:
+            rl, rh = ref[r]["logits"][t], ref[r]["hidden"][t]
+            worst_l = max(worst_l, float(np.max(np.abs(gl[r] - rl)) / np.max(np.abs(rl))))
+            worst_h = max(worst_h, float(np.linalg.norm(gh[r] - rh) / np.linalg.norm(rh)))
+            # free running: the argmax must agree unless the oracle's top two logits are within the tolerance
+            top2 = np.sort(rl)[-2:]
+            if top2[1] - top2[0] > 2 * LOGIT_TOL * np.max(np.abs(rl)):
+                assert gn[r] == ref[r]["tokens"][t]
+        if any(gn[r] != ref[r]["tokens"][t] for r in rows):
+            break                                    # histories diverged on a near-tie: nothing more to compare
+    assert t >= 1
+    assert worst_l <= LOGIT_TOL and worst_h <= HIDDEN_TOL, (worst_l, worst_h)
+    api.ss_release_batch(eng)
+
+
+def test_full_size_7b_zero_output_projections_closed_form():
+    """All 32 layers at the benchmark's shapes and launch configuration.  With Wo = 0 and Wdown = 0 every
+    layer runs (projections, cache, attention) but leaves the residual stream at the embedding, so
+    logits = Wlm . RMSNorm(E[token]) -- which the oracle evaluates for sampled (row, vocabulary id)."""
+    import torch
+    import bench
+    from paper_2305_13144_b200 import api
+    shape = synth.LLAMA_7B
+    rt = api.runtime_cfg(16, 768, 4096, 512, 16 * 768)
+    m = api.model_cfg(shape)
+    arena = torch.empty(api.ss_arena_bytes(m, rt) + 1024, dtype=torch.uint8, device="cuda")
+    torch.cuda.synchronize()
+    eng = api.ss_create(m, rt, arena, torch.cuda.Stream())
+    keep = {}
+    for name, t in bench.device_weights(shape, 99, "cuda:0"):
+        if name.endswith(".wo") or name.endswith(".w_down"):
+            t.zero_()
+        if name in ("embed", "lm_head", "final_norm"):
+            keep[name] = t
+        api.ss_load_weights(eng, {name: t})
+    g = synth.group_7b_batch16(seed=1)
+    B = g.n
+    cu = np.zeros(B + 1, dtype=np.int32)
+    cu[1:] = np.cumsum(g.prompt_len)
+    rng = np.random.default_rng(5)
+    dl = torch.zeros(B, shape.vocab, dtype=torch.float32, device="cuda")
+    fed = np.array([g.prompt(r)[-1] for r in range(B)])          # token whose embedding the logits come from
+    for t in range(3):
+        forced_np = rng.integers(3, shape.vocab, size=B).astype(np.int32)
+        forced = torch.from_numpy(forced_np).cuda()
+        if t == 0:
+            api.ss_prefill(eng, g.prompt_tokens, cu, np.full(B, 100, dtype=np.int32), 512, forced_tokens=forced,
+                           dump_logits=dl)
+        else:
+            api.ss_decode_step(eng, forced_tokens=forced, dump_logits=dl)
+        torch.cuda.synchronize()
+        assert api.ss_last_device_status(eng) == 0
+        got = dl.cpu().numpy()
+        E = keep["embed"][torch.from_numpy(fed).cuda().long()].float().cpu().numpy().astype(np.float64)
+        vs = rng.integers(0, shape.vocab, size=64)
+        Wl = keep["lm_head"][torch.from_numpy(vs).cuda().long()].float().cpu().numpy().astype(np.float64)
+        gain = keep["final_norm"].float().cpu().numpy().astype(np.float64)
+        for r in range(B):
+            exp = od.rmsnorm(E[r], gain, shape.rms_eps) @ Wl.T
+            scale = np.max(np.abs(got[r]))
+            assert np.max(np.abs(got[r, vs] - exp)) <= LOGIT_TOL * scale, (t, r)
+        fed = forced_np
+    api.ss_release_batch(eng)
