@@ -239,7 +239,14 @@ def test_7b_shape_two_layers_sampled_rows():
     """The 7B shape (d 4096, 32 heads x 128, FFN 11008, vocab 32000) cut to two layers, batch 16 with the
     benchmark's prompt lengths; the oracle follows the three rows with the shortest prompts through the
     prompt pass and two decode steps; all rows run free, and a row is compared for as long as its tokens
-    agree with the oracle's (a disagreement is only accepted on a near-tie of the oracle's top two logits)."""
+    agree with the oracle's (a disagreement is only accepted on a near-tie of the oracle's top two logits).
+
+    Hidden-state tolerance here is 2e-2, not the 1e-2 of the small configuration: with N(0, 0.02) weights at
+    d = 4096 the projections' outputs (std ~0.4) dwarf the embedding (std 0.02), so the residual stream's
+    relative error IS the relative error of the bf16 operand chain.  Re-running the oracle's own arithmetic
+    with nothing changed but a round-to-bf16 at the operands the GPU stores in bf16 (normalised input,
+    q/k/v, attention output, SwiGLU output) gives 1.1e-2 on this input, 1.35e-2 with the prompt pass's two
+    extra roundings (q/k/v and gate/up leave its GEMMs as bf16) -- the floor of the format, not of the kernels."""
     import torch
     from paper_2305_13144_b200 import api
     shape = synth.LLAMA_7B.with_layers(2)
@@ -280,7 +287,7 @@ def test_7b_shape_two_layers_sampled_rows():
         if any(gn[r] != ref[r]["tokens"][t] for r in rows):
             break                                    # histories diverged on a near-tie: nothing more to compare
     assert t >= 1
-    assert worst_l <= LOGIT_TOL and worst_h <= HIDDEN_TOL, (worst_l, worst_h)
+    assert worst_l <= LOGIT_TOL and worst_h <= 2e-2, (worst_l, worst_h)
     api.ss_release_batch(eng)
 
 
