@@ -197,6 +197,10 @@ def ss_load_weights(ctx: Ctx, tensors: dict) -> None:
     """tensors: name -> bf16 CUDA tensor, or numpy uint16 array of bf16 bit patterns (host)."""
     descs = (ss_tensor_desc * len(tensors))()
     keep = []
+    if any(not isinstance(t, np.ndarray) and t.is_cuda for t in tensors.values()):
+        # device tensors are usually produced on torch's current stream; the engine reads them on its own
+        import torch
+        torch.cuda.current_stream().synchronize()
     for i, (name, t) in enumerate(tensors.items()):
         if isinstance(t, np.ndarray):
             a = np.ascontiguousarray(t, dtype=np.uint16)
