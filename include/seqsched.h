@@ -116,17 +116,17 @@ typedef struct {
   int32_t n_batches, n_failed;
   float total_ms, prefill_ms, decode_ms;
   double model_bytes;         /* weight + key/value bytes the decode steps had to move         */
-  int64_t kernel_launches;    /* kernels of this library launched (graph nodes counted)        */
+  int64_t kernel_launches;    /* kernels of this library launched                              */
 } ss_group_stats;
 
 /* Bytes of device arena ss_create() needs for this model and capacity. */
 int ss_arena_bytes(const ss_model_cfg* model, const ss_runtime_cfg* rt, size_t* out_bytes);
 
 /* Creates a context.  dev_arena: device memory, 1024-byte aligned, at least ss_arena_bytes().
- * It must outlive the context.  stream: cudaStream_t; ss_decode_steps() and ss_run_group()
- * capture CUDA graphs on it, which the legacy default stream (0) does not allow, so pass a
- * stream created by the caller.  SS_ERR_UNSUPPORTED for shapes the kernels do not cover,
- * SS_ERR_CAPACITY for a short arena. */
+ * It must outlive the context.  stream: cudaStream_t.  A decode step is one cooperative launch
+ * that needs every SM (one CTA per SM waits on grid-wide barriers), so nothing else should occupy
+ * the device while steps run; if the CTAs cannot all be resident the launch fails with SS_ERR_CUDA.
+ * SS_ERR_UNSUPPORTED for shapes the kernels do not cover, SS_ERR_CAPACITY for a short arena. */
 int ss_create(const ss_model_cfg* model, const ss_runtime_cfg* rt, void* dev_arena, size_t arena_bytes,
               void* stream, ss_ctx** out);
 int ss_destroy(ss_ctx* ctx);
@@ -176,7 +176,7 @@ int ss_prefill(ss_ctx* ctx, const int32_t* tokens, const int32_t* cu_seqlens, in
  *                   valid after the stream has been synchronised */
 int ss_decode_step(ss_ctx* ctx, const ss_step_opts* opts, int32_t* next_tokens, int32_t* n_active_host);
 
-/* Replays `n_steps` decode steps from a captured CUDA graph (no options, no per-step outputs). */
+/* Enqueues `n_steps` decode steps back to back (no options, no per-step outputs). */
 int ss_decode_steps(ss_ctx* ctx, int32_t n_steps, int32_t* n_active_host);
 
 /* Copies the batch's results to the host (synchronises the stream).
@@ -246,7 +246,7 @@ const char* ss_strerror(int code);
 int ss_last_device_status(ss_ctx* ctx, uint32_t* out);
 /* Last CUDA error code seen by this context (cudaError_t or CUresult as int). */
 int ss_last_cuda_error(const ss_ctx* ctx);
-/* Kernels launched by this context so far (nodes of replayed graphs counted). */
+/* Kernels launched by this context so far. */
 int64_t ss_kernel_launches(const ss_ctx* ctx);
 
 #ifdef __cplusplus

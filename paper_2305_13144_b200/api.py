@@ -350,8 +350,7 @@ def runtime_cfg(max_batch, max_ctx, max_prefill_tokens, max_new_tokens, kv_pool_
 def make_engine(shape, rt: ss_runtime_cfg, weights: dict, device="cuda:0") -> Ctx:
     """Convenience for tests and the benchmark: allocate the arena with torch, create, load weights.
 
-    The engine gets a stream of its own: CUDA graphs (ss_decode_steps, ss_run_group) cannot be
-    captured on the legacy default stream.  Callers order their own work against it with
+    The engine gets a stream of its own; callers order their own work against it with
     torch.cuda.synchronize() or stream events."""
     import torch
     m = model_cfg(shape)

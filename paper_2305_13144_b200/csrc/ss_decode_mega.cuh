@@ -30,7 +30,6 @@ namespace ss {
 
 constexpr int kMegaThreads = 352;
 constexpr int kMegaWorkers = 256;          // warps 3..10
-constexpr int kMegaAttnChunk = 64;         // cached tokens per attention work item (one warp)
 constexpr int kRowSlice = 512;             // elements of a row handled by one residual work item
 constexpr int kMaxSlices = 16;             // d_model <= 8192
 
@@ -71,10 +70,6 @@ struct MegaArgs {
   bf16 *x, *o, *act;               // GEMM operands: x' [B][d], attention out [B][d], SwiGLU out [B][F]
   float* rowss;                    // [B][kMaxSlices] sums of squares of h per slice
   float* partial;
-  float *part_ml, *part_acc;       // attention partials [B][H][max_chunks][2 | Dh]
-  int32_t* attn_count;             // [B][H] arrival counters (zero between uses)
-  int max_chunks;                  // per row, in units of kMegaAttnChunk
-  int attn_wpp;                    // warps of one CTA that share a (row, head) attention item: 1, 2, 4 or 8
   float* tile_val;
   int32_t* tile_idx;
   int n_tiles_lm;
@@ -251,36 +246,6 @@ __device__ __forceinline__ void stage_inv_rms(const MegaArgs& a, MegaSmem* sm, i
 
 __device__ __forceinline__ void group_bar(int id, int threads) {
   asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
-}
-
-// ---- ahead of the attention stage: pull the cached keys/values it will read into L2 -------------------------
-// Called by the workers while the qkv projection streams its weights (they would otherwise only wait
-// for the accumulators).  Same (row, head) -> warp -> page mapping as stage_attention, one 128-byte
-// line per prefetch, no registers held and nothing to wait for.
-template <int DH>
-__device__ void attention_prefetch(const MegaArgs& a, int wtid, int layer) {
-  const int lane = wtid & 31, wid = wtid >> 5;
-  const int wpp = a.attn_wpp, grp = wid / wpp, wig = wid - grp * wpp, GP = 8 / wpp;
-  const int H = a.H;
-  const uint8_t* kv_layer = reinterpret_cast<const uint8_t*>(a.kv.pool + (size_t)layer * a.kv.layer_stride);
-  const size_t v_off = (size_t)H * kPageTokens * DH * 2;
-  const int n_pairs = a.B * H;
-  for (int p = blockIdx.x * GP + grp; p < n_pairs; p += gridDim.x * GP) {
-    const int r = p / H, hd = p - r * H;
-    if (!a.st.active[r]) continue;
-    const int pos = a.st.ctx_len[r];
-    const int npg = (pos + kPageTokens - 1) / kPageTokens;
-    for (int pi = wig; pi < npg; pi += wpp) {
-      const int pg = a.st.block_table[(size_t)r * a.st.max_pages + pi];
-      if (pg < 0 || pg >= a.kv.n_pages) continue;
-      const int bytes = min(kPageTokens, pos - pi * kPageTokens) * DH * 2;
-      const uint8_t* kb = kv_layer + ((size_t)pg * a.kv.page_elems + (size_t)hd * kPageTokens * DH) * 2;
-      for (int off = lane * 128; off < bytes; off += 32 * 128) {
-        asm volatile("prefetch.global.L2 [%0];" ::"l"(kb + off));
-        asm volatile("prefetch.global.L2 [%0];" ::"l"(kb + v_off + off));
-      }
-    }
-  }
 }
 
 // ---- stage: q,k,v from partials + RoPE + cache append + paged attention ----------------------------------

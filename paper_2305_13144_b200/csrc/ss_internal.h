@@ -21,7 +21,6 @@ int plan_first_pass(const ss_sched_cfg& c, const int32_t* prompt_len, const int3
 constexpr int kPageTokens = 32;        // tokens per key/value page
 constexpr int kTileM = 128;            // weight rows per GEMM tile (tcgen05 M)
 constexpr int kTileK = 64;             // bf16 elements per 128-byte swizzled row
-constexpr int kAttnChunk = 256;        // tokens per decode-attention work item
 constexpr int kMaxBatch = 256;
 
 // Device status codes (which bounded wait expired / which check failed).

@@ -1,11 +1,10 @@
-// Memory-bound kernels of the decode step and the prompt pass (sm_100a).
+// Kernels of the prompt pass, the weight repacking and the batch's first arg-max (sm_100a).
 //
-// Decode (one token per active row):
-//   embed_rmsnorm -> [ qkv GEMM -> rope_append_decode -> attn_decode -> attn_combine -> o GEMM ->
-//   residual_rmsnorm -> gate/up GEMM -> swiglu -> down GEMM -> residual_rmsnorm ] x layers ->
-//   lm_head GEMM -> lmhead_argmax -> bookkeeping
-// The GEMMs leave fp32 partial sums (split along K); the kernel that consumes a projection adds
-// the partials in a fixed order and applies what follows the projection in the model.
+// Prompt pass (all prompt tokens of a chunk at once):
+//   embed_rmsnorm -> [ qkv GEMM -> rope_append_prefill -> attn_prefill -> o GEMM (+= residual) ->
+//   rmsnorm -> gate/up GEMM -> swiglu -> down GEMM (+= residual) -> rmsnorm ] x layers ->
+//   gather_last_rmsnorm -> LM-head GEMM (fp32 partials) -> lmhead_tile_argmax -> bookkeeping
+// The decode step itself is one persistent kernel (ss_decode_mega.cuh) and shares the small helpers here.
 //
 // Every kernel starts with griddepcontrol.launch_dependents / griddepcontrol.wait so that the
 // next kernel's prologue (for a GEMM: its first weight tiles) overlaps this kernel's body.
@@ -108,62 +107,6 @@ embed_rmsnorm_kernel(const int32_t* __restrict__ tokens, const int32_t* __restri
   }
 }
 
-// ------------------------------------------------------------------------------------ RoPE + KV append (decode)
-// grid (H, B), block Dh.  q,k,v come as fp32 partials of the [3d] projection; thread i owns element
-// i of the head.  Pair (i, i+Dh/2) of q and k is rotated by pos * inv_freq[i]; k,v go to the row's page.
-__global__ void __launch_bounds__(128)
-rope_append_decode_kernel(const float* __restrict__ partial, SplitInfo sp, RowState st, KvLayout kv, int layer,
-                          const float* __restrict__ inv_freq, bf16* __restrict__ qbuf, int d, uint32_t* status) {
-  __shared__ float s_q[128], s_k[128];
-  pdl_launch_dependents();
-  pdl_wait();
-  const int hd = blockIdx.x, r = blockIdx.y, i = threadIdx.x;
-  if (!st.active[r]) return;
-  const int Dh = kv.Dh, half = Dh >> 1;
-  const int pos = st.ctx_len[r];
-  const int n = hd * Dh + i;
-  const float qv = sum_partials(partial, sp, n, r);
-  const float kvv = sum_partials(partial, sp, d + n, r);
-  const float vv = sum_partials(partial, sp, 2 * d + n, r);
-  s_q[i] = qv;
-  s_k[i] = kvv;
-  __syncthreads();
-  const int j = i < half ? i : i - half;          // frequency index
-  float sn, cs;
-  sincosf((float)pos * inv_freq[j], &sn, &cs);
-  // first half: x_i cos - x_{i+half} sin; second half: x_i cos + x_{i-half} sin
-  const float qo = i < half ? qv * cs - s_q[i + half] * sn : qv * cs + s_q[i - half] * sn;
-  const float ko = i < half ? kvv * cs - s_k[i + half] * sn : kvv * cs + s_k[i - half] * sn;
-  qbuf[(size_t)r * d + n] = __float2bfloat16_rn(qo);
-  const int page = st.block_table[(size_t)r * st.max_pages + pos / kPageTokens];
-  if (page < 0 || page >= kv.n_pages) {
-    atomicCAS(status, 0u, (uint32_t)kStatusBadPage);
-    return;
-  }
-  bf16* kbase = kv.pool + (size_t)layer * kv.layer_stride + (size_t)page * kv.page_elems +
-                ((size_t)hd * kPageTokens + (pos % kPageTokens)) * Dh;
-  bf16* vbase = kbase + (size_t)kv.H * kPageTokens * Dh;
-  kbase[i] = __float2bfloat16_rn(ko);
-  vbase[i] = __float2bfloat16_rn(vv);
-}
-
-// ------------------------------------------------------------------------------------ decode attention (paged)
-// Work item = (row, head, chunk of kAttnChunk cached tokens); items are dealt round-robin to a
-// fixed grid, so the launch does not depend on the lengths (which live on the device).
-// A group of Dh/8 lanes owns one key: each lane loads 8 bf16 (128 bits) of K and of V, the group
-// reduces q.k with shuffles and keeps a running (max, sum, acc) triple; groups are merged in
-// shared memory and the item's triple goes to the partial buffer.
-struct AttnArgs {
-  RowState st;
-  KvLayout kv;
-  const bf16* q;         // [B][d]
-  float* part_ml;        // [B][H][max_chunks][2]
-  float* part_acc;       // [B][H][max_chunks][Dh]
-  bf16* out;             // [B][d]
-  int B, d, layer, max_chunks;
-  uint32_t* status;
-};
-
 __device__ __forceinline__ void unpack8(const uint4& u, float (&f)[8]) {
   const __nv_bfloat162* p = reinterpret_cast<const __nv_bfloat162*>(&u);
 #pragma unroll
@@ -172,232 +115,6 @@ __device__ __forceinline__ void unpack8(const uint4& u, float (&f)[8]) {
     f[2 * j] = t.x;
     f[2 * j + 1] = t.y;
   }
-}
-
-template <int DH>
-__global__ void __launch_bounds__(128) attn_decode_kernel(AttnArgs a) {
-  constexpr int GROUP = DH / 8;          // lanes per key
-  constexpr int KPW = 32 / GROUP;        // keys per warp
-  constexpr int NG = 4 * KPW;            // groups per CTA
-  constexpr int PPC = kAttnChunk / kPageTokens;
-  __shared__ int s_prefix[kMaxBatch + 1];
-  __shared__ float s_m[NG], s_l[NG];
-  __shared__ float s_acc[NG][DH];
-  __shared__ int s_pages[PPC];
-
-  pdl_launch_dependents();
-  pdl_wait();
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int B = a.B, H = a.kv.H;
-
-  // exclusive prefix of chunk counts over rows (warp 0: 8 rows per lane)
-  if (warp == 0) {
-    int cnt[8], loc = 0;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const int r = lane * 8 + j;
-      int c = 0;
-      if (r < B && a.st.active[r]) c = (a.st.ctx_len[r] + 1 + kAttnChunk - 1) / kAttnChunk;
-      cnt[j] = c;
-      loc += c;
-    }
-    int inc = loc;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int t = __shfl_up_sync(0xffffffffu, inc, o);
-      if (lane >= o) inc += t;
-    }
-    int run = inc - loc;
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      s_prefix[lane * 8 + j] = run;
-      run += cnt[j];
-    }
-    if (lane == 31) s_prefix[kMaxBatch] = inc;
-  }
-  __syncthreads();
-  const int total_chunks = s_prefix[kMaxBatch];
-  const int n_items = total_chunks * H;
-  const int g = warp * KPW + lane / GROUP, gl = lane % GROUP;
-  const float qscale = rsqrtf((float)DH) * 1.4426950408889634f;   // 1/sqrt(Dh) * log2(e)
-  const bf16* kv_layer = a.kv.pool + (size_t)a.layer * a.kv.layer_stride;
-  const size_t v_off = (size_t)H * kPageTokens * DH;
-
-  for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
-    const int cidx = item / H, hd = item - cidx * H;
-    int lo = 0, hi = B - 1;                       // largest r with prefix[r] <= cidx
-    while (lo < hi) {
-      const int mid = (lo + hi + 1) >> 1;
-      if (s_prefix[mid] <= cidx) lo = mid; else hi = mid - 1;
-    }
-    const int r = lo, chunk = cidx - s_prefix[r];
-    const int n_keys = a.st.ctx_len[r] + 1;
-    const int t0 = chunk * kAttnChunk;
-    const int t1 = min(t0 + kAttnChunk, n_keys);
-    if (tid < PPC) {
-      const int pi = t0 / kPageTokens + tid;
-      int pg = 0;
-      if (pi * kPageTokens < t1) {
-        pg = a.st.block_table[(size_t)r * a.st.max_pages + pi];
-        if (pg < 0 || pg >= a.kv.n_pages) { atomicCAS(a.status, 0u, (uint32_t)kStatusBadPage); pg = 0; }
-      }
-      s_pages[tid] = pg;
-    }
-    float q[8];
-    {
-      const uint4 u = *reinterpret_cast<const uint4*>(a.q + (size_t)r * a.d + hd * DH + gl * 8);
-      unpack8(u, q);
-#pragma unroll
-      for (int j = 0; j < 8; ++j) q[j] *= qscale;
-    }
-    __syncthreads();
-
-    float m = -CUDART_INF_F, l = 0.f, acc[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) acc[j] = 0.f;
-
-    constexpr int U = 4;
-    // the trip count is the same for every lane of the warp (the shuffles below need all of them)
-    for (int base = t0; base < t1; base += NG * U) {
-      const int tb = base + g;
-      uint4 kk[U], vv[U];
-      bool valid[U];
-#pragma unroll
-      for (int u = 0; u < U; ++u) {
-        const int t = tb + u * NG;
-        valid[u] = t < t1;
-        kk[u] = make_uint4(0, 0, 0, 0);
-        vv[u] = kk[u];
-        if (valid[u]) {
-          const int pg = s_pages[(t - t0) / kPageTokens];
-          const bf16* kp = kv_layer + (size_t)pg * a.kv.page_elems +
-                           ((size_t)hd * kPageTokens + (t % kPageTokens)) * DH + gl * 8;
-          kk[u] = __ldg(reinterpret_cast<const uint4*>(kp));
-          vv[u] = __ldg(reinterpret_cast<const uint4*>(kp + v_off));
-        }
-      }
-      float s[U];
-#pragma unroll
-      for (int u = 0; u < U; ++u) {
-        float kf[8], dot = 0.f;
-        unpack8(kk[u], kf);
-#pragma unroll
-        for (int j = 0; j < 8; ++j) dot += q[j] * kf[j];
-#pragma unroll
-        for (int o = GROUP / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-        s[u] = valid[u] ? dot : -CUDART_INF_F;
-      }
-      float mn = m;
-#pragma unroll
-      for (int u = 0; u < U; ++u) mn = fmaxf(mn, s[u]);
-      // a group that has seen no key yet keeps (m, l, acc) = (-inf, 0, 0): exp2(-inf - -inf) would be NaN
-      const float sc = (mn == -CUDART_INF_F) ? 1.f : exp2f(m - mn);
-      l *= sc;
-#pragma unroll
-      for (int j = 0; j < 8; ++j) acc[j] *= sc;
-#pragma unroll
-      for (int u = 0; u < U; ++u) {
-        if (valid[u]) {
-          const float pw = exp2f(s[u] - mn);
-          float vf[8];
-          unpack8(vv[u], vf);
-          l += pw;
-#pragma unroll
-          for (int j = 0; j < 8; ++j) acc[j] += pw * vf[j];
-        }
-      }
-      m = mn;
-    }
-    if (gl == 0) { s_m[g] = m; s_l[g] = l; }
-#pragma unroll
-    for (int j = 0; j < 8; ++j) s_acc[g][gl * 8 + j] = acc[j];
-    __syncthreads();
-    if (tid < DH) {
-      float M = -CUDART_INF_F;
-#pragma unroll
-      for (int x = 0; x < NG; ++x) M = fmaxf(M, s_m[x]);
-      float L = 0.f, A = 0.f;
-#pragma unroll
-      for (int x = 0; x < NG; ++x) {
-        const float w = (s_m[x] == -CUDART_INF_F) ? 0.f : exp2f(s_m[x] - M);
-        L += s_l[x] * w;
-        A += s_acc[x][tid] * w;
-      }
-      const size_t slot = ((size_t)r * H + hd) * a.max_chunks + chunk;
-      a.part_acc[slot * DH + tid] = A;
-      if (tid == 0) { a.part_ml[slot * 2] = M; a.part_ml[slot * 2 + 1] = L; }
-    }
-    __syncthreads();
-  }
-}
-
-// grid (H, B), block DH: merge the chunks of one (row, head); out = acc / sum in bf16.
-template <int DH>
-__global__ void __launch_bounds__(DH) attn_combine_kernel(AttnArgs a) {
-  pdl_launch_dependents();
-  pdl_wait();
-  const int hd = blockIdx.x, r = blockIdx.y, i = threadIdx.x;
-  if (!a.st.active[r]) return;
-  const int n_keys = a.st.ctx_len[r] + 1;
-  const int nch = (n_keys + kAttnChunk - 1) / kAttnChunk;
-  const size_t base = ((size_t)r * a.kv.H + hd) * a.max_chunks;
-  float M = -CUDART_INF_F;
-  for (int c = 0; c < nch; ++c) M = fmaxf(M, a.part_ml[(base + c) * 2]);
-  float L = 0.f, A = 0.f;
-  for (int c = 0; c < nch; ++c) {
-    const float w = exp2f(a.part_ml[(base + c) * 2] - M);
-    L += a.part_ml[(base + c) * 2 + 1] * w;
-    A += a.part_acc[(base + c) * DH + i] * w;
-  }
-  a.out[(size_t)r * a.d + hd * DH + i] = __float2bfloat16_rn(A / L);
-}
-
-// ------------------------------------------------------------------------------------ residual + RMSNorm (decode)
-// h[r] += projection (from partials); x[r] = RMSNorm(h[r]) * g.  grid B, block 1024 (d <= 8192).
-__global__ void __launch_bounds__(1024)
-residual_rmsnorm_partial_kernel(const float* __restrict__ partial, SplitInfo sp, const int32_t* __restrict__ active,
-                                float* __restrict__ h, const bf16* __restrict__ g, bf16* __restrict__ x,
-                                float* __restrict__ dump_hidden, int d, float eps) {
-  __shared__ float red[32];
-  pdl_launch_dependents();
-  pdl_wait();
-  const int r = blockIdx.x;
-  if (active && !active[r]) return;
-  constexpr int kMaxPer = 8;
-  float v[kMaxPer];
-  float ss = 0.f;
-#pragma unroll
-  for (int c = 0; c < kMaxPer; ++c) {
-    const int i = threadIdx.x + c * 1024;
-    v[c] = 0.f;
-    if (i < d) {
-      v[c] = h[(size_t)r * d + i] + sum_partials(partial, sp, i, r);
-      ss += v[c] * v[c];
-    }
-  }
-  ss = block_sum(ss, red);
-  const float inv = rsqrtf(ss / d + eps);
-#pragma unroll
-  for (int c = 0; c < kMaxPer; ++c) {
-    const int i = threadIdx.x + c * 1024;
-    if (i < d) {
-      h[(size_t)r * d + i] = v[c];
-      if (dump_hidden) dump_hidden[(size_t)r * d + i] = v[c];
-      x[(size_t)r * d + i] = __float2bfloat16_rn(v[c] * inv * __bfloat162float(g[i]));
-    }
-  }
-}
-
-// act[r][f] = silu(gate) * up from the partials of the stacked [2F] projection.  grid (ceil(F/256), B)
-__global__ void __launch_bounds__(256)
-swiglu_partial_kernel(const float* __restrict__ partial, SplitInfo sp, bf16* __restrict__ act, int F) {
-  pdl_launch_dependents();
-  pdl_wait();
-  const int r = blockIdx.y, f = blockIdx.x * blockDim.x + threadIdx.x;
-  if (f >= F) return;
-  const float gt = sum_partials(partial, sp, f, r);
-  const float up = sum_partials(partial, sp, F + f, r);
-  act[(size_t)r * F + f] = __float2bfloat16_rn(gt / (1.f + __expf(-gt)) * up);
 }
 
 // ------------------------------------------------------------------------------------ LM head argmax

@@ -96,8 +96,6 @@ struct ss_ctx {
   bool use_pdl = true;
   int last_cuda = 0;
   int64_t launches = 0;
-  bool capturing = false;
-  int64_t capture_count = 0;
   EncodeTiledFn encode = nullptr;
 
   // ---- arena
@@ -123,14 +121,11 @@ struct ss_ctx {
   bf16 *x = nullptr, *qkv = nullptr, *attn_o = nullptr, *gu = nullptr, *act = nullptr;
   // decode activations (kMaxBatch rows)
   float* h_dec = nullptr;
-  bf16 *x_dec = nullptr, *q_dec = nullptr, *o_dec = nullptr, *act_dec = nullptr;
+  bf16 *x_dec = nullptr, *o_dec = nullptr, *act_dec = nullptr;
   float* partial = nullptr;
   size_t partial_bytes = 0;
-  float *part_ml = nullptr, *part_acc = nullptr;
-  int max_chunks = 0;
   TileSeg* tbl[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};   // qkv, o, gate/up, down, lm head
   float* rowss = nullptr;          // [kMaxBatch][kMaxSlices]
-  int32_t* attn_count = nullptr;   // [kMaxBatch][H]
   unsigned long long* grid_ctr = nullptr;
   unsigned long long* trace = nullptr;  // stage-boundary time stamps of the last decode step
   int trace_len = 0;
@@ -153,8 +148,6 @@ struct ss_ctx {
   bool in_batch = false;
   std::vector<int32_t> prompt_len;
   int32_t* pinned = nullptr;     // [0] n_active, [1] status
-  std::map<int, cudaGraphExec_t> graphs;   // decode step per batch size
-  int64_t graph_nodes = 0;
 };
 
 namespace {
@@ -181,7 +174,7 @@ cudaError_t launch(ss_ctx* c, void (*kern)(KArgs...), dim3 grid, dim3 block, siz
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = c->use_pdl ? 1 : 0;
-  if (c->capturing) c->capture_count++; else c->launches++;
+  c->launches++;
   return cudaLaunchKernelEx(&cfg, kern, KArgs(args)...);
 }
 
@@ -259,10 +252,10 @@ struct Offsets {
   size_t embed, lm_head, final_norm, staging, staging_bytes, weights_end;
   std::vector<size_t> attn_norm, wqkv, wo, ffn_norm, wgu, wdown;
   size_t inv_freq, status, rows, block_table, out_tokens, tok, h, x, qkv, attn_o, gu, act;
-  size_t h_dec, x_dec, q_dec, o_dec, act_dec, partial, part_ml, part_acc, kv;
-  size_t tbl[5], tile_val, tile_idx, rowss, attn_count, grid_ctr, wptr, norm_ptr, trace;
+  size_t h_dec, x_dec, o_dec, act_dec, partial, kv;
+  size_t tbl[5], tile_val, tile_idx, rowss, grid_ctr, wptr, norm_ptr, trace;
   size_t partial_bytes;
-  int R, max_pages, n_pages, max_chunks;
+  int R, max_pages, n_pages;
   size_t total;
 };
 
@@ -313,7 +306,6 @@ void layout(const ss_model_cfg& m, const ss_runtime_cfg& rt, int n_sm, Offsets& 
   o.act = a.take((size_t)o.R * F * 2);
   o.h_dec = a.take((size_t)kMaxBatch * d * 4);
   o.x_dec = a.take((size_t)kMaxBatch * d * 2);
-  o.q_dec = a.take((size_t)kMaxBatch * d * 2);
   o.o_dec = a.take((size_t)kMaxBatch * d * 2);
   o.act_dec = a.take((size_t)kMaxBatch * F * 2);
   // partial work space: the largest decode GEMM at the widest token tile
@@ -326,15 +318,11 @@ void layout(const ss_model_cfg& m, const ss_runtime_cfg& rt, int n_sm, Offsets& 
   }
   o.partial_bytes = pb;
   o.partial = a.take(pb);
-  o.max_chunks = ceil_div(rt.max_ctx, kMegaAttnChunk);
   o.rowss = a.take((size_t)kMaxBatch * kMaxSlices * 4);
-  o.attn_count = a.take((size_t)kMaxBatch * m.n_heads * 4);
   o.grid_ctr = a.take(64);
   o.wptr = a.take((size_t)(4 * m.n_layers + 1) * sizeof(void*));
   o.norm_ptr = a.take((size_t)(2 * m.n_layers + 1) * sizeof(void*));
   o.trace = a.take((size_t)(2 + 4 * (4 * m.n_layers + 1)) * 8);
-  o.part_ml = a.take((size_t)kMaxBatch * m.n_heads * o.max_chunks * 2 * 4);
-  o.part_acc = a.take((size_t)kMaxBatch * m.n_heads * o.max_chunks * m.head_dim * 4);
   for (int i = 0; i < 5; ++i) o.tbl[i] = a.take((size_t)ceil_div(shapes[i][0], kTileM) * sizeof(TileSeg));
   o.tile_val = a.take((size_t)kMaxBatch * ceil_div((int)V, kTileM) * 4);
   o.tile_idx = a.take((size_t)kMaxBatch * ceil_div((int)V, kTileM) * 4);
@@ -430,14 +418,6 @@ int enqueue_decode_step(ss_ctx* c, const ss_step_opts* opts, int32_t* next_token
   a.st = c->st; a.kv = c->kv;
   a.h = c->h_dec; a.x = c->x_dec; a.o = c->o_dec; a.act = c->act_dec;
   a.rowss = c->rowss; a.partial = c->partial;
-  {
-    // one round over the worker-warp groups when the items allow it (the per-item set-up is latency-bound)
-    const long long pairs = (long long)B * m.n_heads;
-    int wpp = 8;
-    while (wpp > 1 && pairs * wpp > 1LL * c->n_sm * 8) wpp >>= 1;
-    a.attn_wpp = wpp;
-  }
-  a.part_ml = c->part_ml; a.part_acc = c->part_acc; a.attn_count = c->attn_count; a.max_chunks = c->max_chunks;
   a.tile_val = c->tile_val; a.tile_idx = c->tile_idx; a.n_tiles_lm = c->n_tiles_lm;
   a.forced = opts ? opts->forced_tokens : nullptr;
   a.next_tokens = next_tokens;
@@ -602,16 +582,11 @@ int ss_create(const ss_model_cfg* model, const ss_runtime_cfg* rt, void* dev_are
   c->act = (bf16*)(A + o.act);
   c->h_dec = (float*)(A + o.h_dec);
   c->x_dec = (bf16*)(A + o.x_dec);
-  c->q_dec = (bf16*)(A + o.q_dec);
   c->o_dec = (bf16*)(A + o.o_dec);
   c->act_dec = (bf16*)(A + o.act_dec);
   c->partial = (float*)(A + o.partial);
   c->partial_bytes = o.partial_bytes;
-  c->part_ml = (float*)(A + o.part_ml);
-  c->part_acc = (float*)(A + o.part_acc);
-  c->max_chunks = o.max_chunks;
   c->rowss = (float*)(A + o.rowss);
-  c->attn_count = (int32_t*)(A + o.attn_count);
   c->grid_ctr = (unsigned long long*)(A + o.grid_ctr);
   c->wptr_dev = (const uint8_t**)(A + o.wptr);
   c->trace = (unsigned long long*)(A + o.trace);
@@ -682,7 +657,6 @@ int ss_create(const ss_model_cfg* model, const ss_runtime_cfg* rt, void* dev_are
 int ss_destroy(ss_ctx* c) {
   if (!c) return SS_ERR_ARG;
   cudaStreamSynchronize(c->stream);
-  for (auto& g : c->graphs) cudaGraphExecDestroy(g.second);
   if (c->pinned) cudaFreeHost(c->pinned);
   delete c;
   return SS_OK;
@@ -866,9 +840,8 @@ int ss_read_batch(ss_ctx* c, int32_t* out_tokens, int32_t stride, int32_t* out_l
   SS_CUDA(c, cudaMemcpyAsync(c->pinned + 1, c->status, 4, cudaMemcpyDeviceToHost, c->stream));
   SS_CUDA(c, cudaStreamSynchronize(c->stream));
   if (c->pinned[1] != 0) {
-    // an aborted step leaves the grid-barrier counter and the arrival counters in an unknown state
+    // an aborted step leaves the grid-barrier counter in an unknown state
     cudaMemsetAsync(c->grid_ctr, 0, 8, c->stream);
-    cudaMemsetAsync(c->attn_count, 0, (size_t)kMaxBatch * c->m.n_heads * 4, c->stream);
     cudaStreamSynchronize(c->stream);
     c->grid_epochs = 0;
     return c->pinned[1] == (int32_t)kStatusBadPage ? SS_ERR_STATE : SS_ERR_DEVICE_TIMEOUT;
