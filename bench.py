@@ -39,6 +39,10 @@ from paper_2305_13144_b200 import synth  # noqa: E402
 METRIC = "generated tokens/s"
 WORKLOAD = "llama7b-shape bf16, one vanilla micro-batch of 16, prompts U[64,256], responses lognormal(120,0.7)<=512"
 FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one decode-step launch, from the ncu captures summarised in
+# profiles/decode_step_mega_7b_shape_ncu_full.md (2- and 4-layer cases, scaled to 32 layers).  Set to None
+# whenever the kernel changes after the capture.
+TRAFFIC_BYTES_PER_DECODE_STEP = None
 
 
 def measured_peaks():
@@ -205,6 +209,34 @@ def aggregate(tokens_local: float, seconds_local: float, dist):
     return float(t.item()), float(s.item())
 
 
+def stage_trace(eng, api, g, steps=60):
+    """Where one decode step spends its time: the batch's prompt pass, `steps` decode steps, then the stage
+    stamps of the last step (ss_step_trace), averaged per projection type (microseconds)."""
+    import torch
+    cu = np.zeros(g.n + 1, dtype=np.int32)
+    cu[1:] = np.cumsum(g.prompt_len)
+    api.ss_prefill(eng, g.prompt_tokens, cu, g.true_len, 512)
+    api.ss_decode_steps(eng, steps)
+    torch.cuda.synchronize()
+    tr = api.ss_step_trace(eng).astype(np.int64)
+    api.ss_release_batch(eng)
+    tr = tr - tr[0]
+    ev = tr[2:].reshape(-1, 4)
+    names = ["qkv", "o", "gate_up", "down"]
+    acc, cnt, prev = {}, {}, tr[1]
+    for i, row in enumerate(ev):
+        nm = "lm_head" if i == len(ev) - 1 else names[i % 4]
+        d = np.array([row[0] - prev, row[1] - row[0], row[2] - row[1], row[3] - row[2]], dtype=np.float64)
+        prev = row[3]
+        acc[nm] = acc.get(nm, 0) + d
+        cnt[nm] = cnt.get(nm, 0) + 1
+    out = {"step_us": float(tr[-1]) / 1e3, "after_steps": steps,
+           "columns": ["projection_and_drain", "barrier", "following_stage", "barrier"]}
+    for nm in acc:
+        out[nm] = [round(float(x) / cnt[nm] / 1e3, 2) for x in acc[nm]]
+    return out
+
+
 def run_group_arm(eng, api, g, cfg, perm):
     t0 = time.time()
     res = api.ss_run_group(eng, cfg, g.prompt_tokens, g.prompt_off, g.pred_len, perm, g.true_len)
@@ -228,6 +260,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--group-arms", action="store_true", help="also run the 1024-query group: vanilla vs scheduled")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--trace", action="store_true", help="add the per-stage timing of one decode step")
     ap.add_argument("--layers", type=int, default=0, help="debug: truncate the model (invalidates the number)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
@@ -310,13 +343,15 @@ def main():
             "gpu_launches": int(launches),
             "roofline": {"bound": "hbm", "kernel": "decode_step_mega_kernel (one persistent cooperative launch per decode step)",
                          "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "peak_source": which, "traffic": None,
+                         "peak_source": which, "traffic": TRAFFIC_BYTES_PER_DECODE_STEP if shape.n_layers == 32 else None,
                          "ms_per_decode_step": decode_s / max(1, steps_dec) * 1e3,
                          "bytes_per_decode_step": model_bytes / max(1, steps_dec)},
             "phases": {"prefill_s_per_step": prefill_s / args.steps, "decode_s_per_step": decode_s / args.steps,
                        "decode_steps_per_step": steps_dec / args.steps},
             "clocks": clk.summary(),
         }
+        if args.trace:
+            line["stage_trace"] = stage_trace(eng, api, g)
         if args.group_arms:
             g3 = synth.group_7b_1024(seed=0)
             arms = {}
