@@ -104,6 +104,11 @@ struct MegaSmem {
   __align__(16) float q_s[8][128]; // attention: per worker warp, rotated query (then the new token's value); read as float4
   __align__(16) float att_s[8][9][132];   // attention: [pair of the pass][partial: 8 warps + new token][acc[Dh], max, sum]
   int pair_id[8], pair_ustart[9], pair_n, pair_next, pair_lo, pair_hi;
+  // per-step attention set-up that does not change from layer to layer (valid when att_single)
+  int att_single;                  // the CTA's pairs fit one pass: the lists above are built once per step
+  int pair_pos[8], pair_pgnew[8];  // new token's position and page
+  int unit_pg[8][8];               // page ids of each warp's units (when it has at most 8)
+  float rope_c[8][128], rope_sn[8][128];   // cos / sin of the new position per pair, cooperative lane layout
   float red[8];
   uint32_t am_key[2][4][64];       // per-tile arg-max scratch: [tile half][warp][batch row]
   int am_id[2][4][64];
@@ -285,21 +290,14 @@ __device__ __forceinline__ void sum_partialsN_cg(const float* __restrict__ parti
 constexpr int kAttnPass = 8;               // pairs per pass (= worker warps)
 constexpr int kAttnSlots = 9;              // partials per pair: one per warp + the new token
 
+// Once per step (the lengths do not change between layers): pages per row, this CTA's run of pairs, and --
+// when the run fits one pass -- the pass list, the new tokens' positions/pages/rotations and the page ids
+// of every warp's units.
 template <int DH>
-__device__ void stage_attention(const MegaArgs& a, MegaSmem* sm, int wtid, int layer) {
-  constexpr int GROUP = DH / 32;           // lanes per key in the cache scan
-  constexpr int KPW = 32 / GROUP;          // keys per warp-wide load step
-  constexpr int EPL = DH / 32;             // cooperative layout: consecutive dimensions per lane
-  constexpr int STEPS = kPageTokens / KPW; // load steps per page (4 at Dh 128, 2 at Dh 64)
-  constexpr int U = 2;                     // load steps per batch
+__device__ void attention_setup(const MegaArgs& a, MegaSmem* sm, int wtid) {
+  constexpr int EPL = DH / 32;
   const int lane = wtid & 31, wid = wtid >> 5;
-  const int gl = lane % GROUP, g = lane / GROUP;
-  const int H = a.H, d = a.d, B = a.B;
-  const MegaGemmShape& gs = a.shape[0];
-  const float qscale = rsqrtf((float)DH) * 1.4426950408889634f;
-  const bf16* kv_layer = a.kv.pool + (size_t)layer * a.kv.layer_stride;
-  const size_t v_off = (size_t)H * kPageTokens * DH;
-
+  const int H = a.H, B = a.B;
   // ---- pages per row (exclusive prefix, active rows only) and this CTA's run of pairs
   if (wid == 0) {
     int cnt[8], loc = 0;
@@ -341,11 +339,77 @@ __device__ void stage_attention(const MegaArgs& a, MegaSmem* sm, int wtid, int l
     if (mylo <= myhi) { atomicMin(&sm->pair_lo, mylo); atomicMax(&sm->pair_hi, myhi); }
   }
   named_bar_workers();
+  const int p_begin = sm->pair_lo, p_end = sm->pair_hi + 1;
+  if (wid == 0) {
+    int n = 0, p = p_begin, ustart = 0;
+    while (p < p_end && n < kAttnPass) {
+      const int r = p / H;
+      const int npr = sm->prefix[r + 1] - sm->prefix[r];
+      if (npr <= 0) { p = (r + 1) * H; continue; }
+      if (lane == 0) { sm->pair_id[n] = p; sm->pair_ustart[n] = ustart; }
+      ustart += npr;
+      ++n;
+      ++p;
+    }
+    // any pair with work left beyond the first eight?
+    bool more = false;
+    for (int q = p; q < p_end && !more; ) {
+      const int r = q / H;
+      if (sm->prefix[r + 1] - sm->prefix[r] > 0) more = true; else q = (r + 1) * H;
+    }
+    if (lane == 0) { sm->pair_n = n; sm->pair_next = p; sm->pair_ustart[n] = ustart; sm->att_single = more ? 0 : 1; }
+  }
+  named_bar_workers();
+  if (sm->att_single) {
+    const int np = sm->pair_n, U = sm->pair_ustart[np];
+    if (wid < np) {
+      const int p = sm->pair_id[wid];
+      const int r = p / H;
+      const int pos = a.st.ctx_len[r];
+#pragma unroll
+      for (int j = 0; j < EPL; ++j) {
+        float sn, cs;
+        sincosf((float)pos * a.inv_freq[(lane & 15) * EPL + j], &sn, &cs);
+        sm->rope_c[wid][lane * EPL + j] = cs;
+        sm->rope_sn[wid][lane * EPL + j] = sn;
+      }
+      if (lane == 0) {
+        sm->pair_pos[wid] = pos;
+        sm->pair_pgnew[wid] = a.st.block_table[(size_t)r * a.st.max_pages + pos / kPageTokens];
+      }
+    }
+    const int u0 = (int)((long long)wid * U / 8), u1 = (int)((long long)(wid + 1) * U / 8);
+    if (lane < 8 && u0 + lane < u1) {
+      const int u = u0 + lane;
+      int j = 0;
+      while (j + 1 < np && sm->pair_ustart[j + 1] <= u) ++j;
+      sm->unit_pg[wid][lane] = a.st.block_table[(size_t)(sm->pair_id[j] / H) * a.st.max_pages + (u - sm->pair_ustart[j])];
+    }
+  }
+  named_bar_workers();
+}
+
+template <int DH>
+__device__ void stage_attention(const MegaArgs& a, MegaSmem* sm, int wtid, int layer) {
+  constexpr int GROUP = DH / 32;           // lanes per key in the cache scan
+  constexpr int KPW = 32 / GROUP;          // keys per warp-wide load step
+  constexpr int EPL = DH / 32;             // cooperative layout: consecutive dimensions per lane
+  constexpr int STEPS = kPageTokens / KPW; // load steps per page (4 at Dh 128, 2 at Dh 64)
+  constexpr int U = 2;                     // load steps per batch
+  const int lane = wtid & 31, wid = wtid >> 5;
+  const int gl = lane % GROUP, g = lane / GROUP;
+  const int H = a.H, d = a.d, B = a.B;
+  const MegaGemmShape& gs = a.shape[0];
+  const float qscale = rsqrtf((float)DH) * 1.4426950408889634f;
+  const bf16* kv_layer = a.kv.pool + (size_t)layer * a.kv.layer_stride;
+  const size_t v_off = (size_t)H * kPageTokens * DH;
+
   const int p_begin = sm->pair_lo, p_end = sm->pair_hi + 1;          // empty run: lo > hi
+  const bool single = sm->att_single != 0;
 
   for (int pass0 = p_begin; pass0 < p_end; ) {
     // ---- the pass: next (up to 8) pairs with work; pair_id / pair_pages / pair_ustart in shared memory
-    if (wid == 0) {
+    if (wid == 0 && !single) {
       int n = 0, p = pass0, ustart = 0;
       // lanes walk the pairs together (few iterations: rows without work are skipped by whole rows)
       while (p < p_end && n < kAttnPass) {
@@ -368,17 +432,20 @@ __device__ void stage_attention(const MegaArgs& a, MegaSmem* sm, int wtid, int l
     if (wid < np_pass) {
       const int p = sm->pair_id[wid];
       const int r = p / H, hd = p - r * H;
-      const int pos = a.st.ctx_len[r];
+      const int pos = single ? sm->pair_pos[wid] : a.st.ctx_len[r];
       const float inv = row_inv_rms(a, r);
       const int e0 = lane * EPL;
       float sn[EPL], cs[EPL];
 #pragma unroll
-      for (int j = 0; j < EPL; ++j) sincosf((float)pos * a.inv_freq[(lane & 15) * EPL + j], &sn[j], &cs[j]);
+      for (int j = 0; j < EPL; ++j) {
+        if (single) { cs[j] = sm->rope_c[wid][e0 + j]; sn[j] = sm->rope_sn[wid][e0 + j]; }
+        else sincosf((float)pos * a.inv_freq[(lane & 15) * EPL + j], &sn[j], &cs[j]);
+      }
       float qx[EPL], kx[EPL], vx[EPL];
       sum_partialsN_cg<EPL>(a.partial, gs, a.NT, hd * DH + e0, r, qx);
       sum_partialsN_cg<EPL>(a.partial, gs, a.NT, d + hd * DH + e0, r, kx);
       sum_partialsN_cg<EPL>(a.partial, gs, a.NT, 2 * d + hd * DH + e0, r, vx);
-      int pg = a.st.block_table[(size_t)r * a.st.max_pages + pos / kPageTokens];
+      int pg = single ? sm->pair_pgnew[wid] : a.st.block_table[(size_t)r * a.st.max_pages + pos / kPageTokens];
       if (pg < 0 || pg >= a.kv.n_pages) { atomicCAS(a.status, 0u, (uint32_t)kStatusBadPage); pg = -1; }
       bf16* kdst = a.kv.pool + (size_t)layer * a.kv.layer_stride + (size_t)(pg < 0 ? 0 : pg) * a.kv.page_elems +
                    ((size_t)hd * kPageTokens + (pos % kPageTokens)) * DH + e0;
@@ -446,8 +513,8 @@ __device__ void stage_attention(const MegaArgs& a, MegaSmem* sm, int wtid, int l
         const int p = sm->pair_id[j];
         const int r = p / H, hd = p - r * H;
         const int pi = u - sm->pair_ustart[j];
-        const int pos = a.st.ctx_len[r];
-        int pg = a.st.block_table[(size_t)r * a.st.max_pages + pi];
+        const int pos = single ? sm->pair_pos[j] : a.st.ctx_len[r];
+        int pg = (single && u - u0 < 8) ? sm->unit_pg[wid][u - u0] : a.st.block_table[(size_t)r * a.st.max_pages + pi];
         if (pg < 0 || pg >= a.kv.n_pages) { atomicCAS(a.status, 0u, (uint32_t)kStatusBadPage); pg = 0; }
         const int tcount = min(kPageTokens, pos - pi * kPageTokens);
         const bf16* kb = kv_layer + (size_t)pg * a.kv.page_elems + (size_t)hd * kPageTokens * DH;
@@ -539,7 +606,7 @@ __device__ void stage_attention(const MegaArgs& a, MegaSmem* sm, int wtid, int l
 #pragma unroll
       for (int j = 0; j < EPL; ++j) a.o[(size_t)r * d + hd * DH + e0 + j] = __float2bfloat16_rn(A[j] * il);
     }
-    pass0 = sm->pair_next;
+    pass0 = single ? p_end : sm->pair_next;       // a single pass covers the whole run
     named_bar_workers();
   }
 }
@@ -831,6 +898,7 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
     int tr = 0;
     if (tracer) a.trace[tr++] = global_timer_ns();
     if (cta == 0 && wtid == 0) a.st.scalars[1] = 0;   // rows still active after this step (counted in the last stage)
+    attention_setup<DH>(a, sm, wtid);
     stage_residual(a, sm, wtid, 0, nullptr, a.norm_ptr[0], a.n_layers == 0);
     ok = grid_barrier(a, sm, epoch, wtid);
     if (ok && wtid == 0) sm->act_epoch = 1;
