@@ -252,6 +252,26 @@ def run_group_arm(eng, api, g, cfg, perm):
             "decode_gbs": st["model_bytes"] / (st["decode_ms"] / 1e3) / 1e9 if st["decode_ms"] > 0 else None}
 
 
+def run_group_13b(api, device):
+    """Configuration 5: LLaMA-13B shape, 512 queries, prompts U[64,512], responses lognormal(200, 0.7) <= 2048,
+    predicted = true + N(0,40), bins of 50; vanilla batching vs FCR + variable batch size in a 120 GB KV budget."""
+    shape = synth.LLAMA_13B
+    kv_tok = 2 * shape.d_model * 2 * shape.n_layers
+    rt = api.runtime_cfg(256, 512 + 2048, 16384, 2048, int(120e9 // kv_tok))
+    eng = make_engine(shape, rt, seed=4321, device=device)
+    g = synth.group_13b_512(seed=0)
+    arms = {}
+    arms["vanilla"] = run_group_arm(eng, api, g, api.sched_cfg(vanilla=True, max_new_tokens=2048),
+                                    synth.make_permutation(g.n, 0))
+    arms["scheduled_fcr_vbs"] = run_group_arm(
+        eng, api, g, api.sched_cfg(use_vbs=True, max_new_tokens=2048, kv_budget_bytes=int(120e9),
+                                   kv_bytes_per_token=kv_tok), None)
+    arms["scheduled_fcr_vbs"]["gain_vs_vanilla"] = arms["scheduled_fcr_vbs"]["tokens_per_s"] / arms["vanilla"]["tokens_per_s"]
+    return {"metric": METRIC, "unit": "tokens/s", "n_gpus": 1, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "llama13b-shape bf16, 512 queries, prompts U[64,512], responses lognormal(200,0.7)<=2048"},
+            "value": arms["scheduled_fcr_vbs"]["tokens_per_s"], "arms": arms}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -261,6 +281,8 @@ def main():
     ap.add_argument("--group-arms", action="store_true", help="also run the 1024-query group: vanilla vs scheduled")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--trace", action="store_true", help="add the per-stage timing of one decode step")
+    ap.add_argument("--group-13b", action="store_true",
+                    help="instead of the batch-16 workload: the 13B-shape group of 512 queries, vanilla vs scheduled")
     ap.add_argument("--layers", type=int, default=0, help="debug: truncate the model (invalidates the number)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
@@ -283,6 +305,10 @@ def main():
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=torch.device(device))
 
+    if args.group_13b:
+        if rank == 0:
+            print(json.dumps(run_group_13b(api, device)), flush=True)
+        return
     shape = synth.LLAMA_7B if not args.layers else synth.LLAMA_7B.with_layers(args.layers)
     kv_tok = 2 * shape.d_model * 2 * shape.n_layers
     if args.group_arms:
