@@ -144,8 +144,9 @@ __device__ __forceinline__ bool grid_barrier(const MegaArgs& a, MegaSmem* sm, un
   named_bar_workers();
   ++epoch;
   if (wtid == 0) {
-    __threadfence();
-    atomicAdd(a.grid_ctr, 1ULL);
+    // arrive: release-add without waiting for the old value (the writes of the whole CTA, seen through the
+    // bar.sync above, are ordered before it); then poll with acquire loads
+    asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(a.grid_ctr), "l"(1ULL) : "memory");
     const unsigned long long target = a.grid_base + epoch * gridDim.x;
     const long long t0 = clock64();
     while (ld_acquire_u64(a.grid_ctr) < target) {
@@ -156,7 +157,6 @@ __device__ __forceinline__ bool grid_barrier(const MegaArgs& a, MegaSmem* sm, un
         break;
       }
     }
-    __threadfence();
   }
   named_bar_workers();
   return sm->abort == 0;
