@@ -10,7 +10,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libseqsched.so")
 SOURCES = ["ss_runtime.cu", "ss_noalloc.cu", "ss_sched.cpp"]
-HEADERS = ["ss_internal.h", "ss_gemm.cuh", "ss_kernels.cuh"]
+HEADERS = ["ss_internal.h", "ss_gemm.cuh", "ss_kernels.cuh", "ss_decode_mega.cuh"]
 
 
 def _stale() -> bool:

@@ -8,13 +8,19 @@
 // stage, the ring keeps filling with the next projection's weights.
 //
 // Warp roles (352 threads):
-//   warp 0      weight producer: linear bulk copies of 16 KiB (tile, k-block) images into the ring
+//   warp 0      weight producer: linear bulk copies of 32 KiB (256-row tile, k-block) images into the ring
 //   warp 1      MMA issuer: tcgen05.mma, accumulators in tensor memory (two buffers)
-//   warp 2      activation loader: TMA loads of the [NT x 64] activation block of each ring stage,
+//   warp 2      activation loader: TMA loads of the [tokens x 64] activation block of each ring stage,
 //               issued once the stage that produced the activations has passed its grid barrier
 //   warps 3-10  workers: drain accumulators to fp32 partials, then run the stage between two
 //               projections (partial sums in CTA order, RoPE, cache append, attention, residual,
 //               SwiGLU, arg-max, bookkeeping), separated by grid barriers
+//
+// Operand roles: one tcgen05.mma costs about the same issue time whatever its shape, so the decode
+// projections put the WEIGHTS on the wide side: D[token, row] += X[token, 16] . W[row, 16]^T with
+// M = 128 token lanes and N = 256 weight rows (8 KiB of weights per instruction).  Token lanes
+// beyond the batch compute on whatever shared memory follows the activation block; rows of D are
+// independent, and those lanes are never read.
 //
 // RMSNorm is applied lazily: the residual stage writes x' = bf16(h * g) and per-slice sums of
 // squares; since a projection is linear, the consumer of its partial sums multiplies by
@@ -62,7 +68,9 @@ struct MegaArgs {
   const float* inv_freq;
   MegaGemmShape shape[5];          // qkv, o, gate/up, down, lm head
   // batch
-  int B, NT, stages, tmem_cols;
+  int B, NT, stages;
+  int m_tiles;                     // 128-token accumulator tiles (1, or 2 above 128 rows)
+  int x_rows;                      // activation rows per TMA load (the tensor map's box height)
   RowState st;
   KvLayout kv;
   // activations (decode buffers)
@@ -164,9 +172,9 @@ __device__ __forceinline__ bool grid_barrier(const MegaArgs& a, MegaSmem* sm, un
 
 // Sum of the partials of output row n for token tok (CTA order), read past L1.
 __device__ __forceinline__ float sum_partials_cg(const float* __restrict__ partial, const MegaGemmShape& s, int NT, int n, int tok) {
-  const int4 t = __ldg(reinterpret_cast<const int4*>(s.tiles) + (n >> 7));
-  const size_t slot_stride = (size_t)NT * 128;
-  const size_t off = (size_t)tok * 128 + (n & 127);
+  const int4 t = __ldg(reinterpret_cast<const int4*>(s.tiles) + n / kTileN);
+  const size_t slot_stride = (size_t)NT * kTileN;
+  const size_t off = (size_t)tok * kTileN + (n % kTileN);
   float acc = __ldcg(partial + (size_t)t.x * slot_stride + off);
   const size_t cta_stride = slot_stride * s.max_seg;
   for (int c = t.y; c <= t.z; ++c) acc += __ldcg(partial + (size_t)c * cta_stride + off);
@@ -228,9 +236,9 @@ __device__ void stage_residual(const MegaArgs& a, MegaSmem* sm, int wtid, int mo
 // 8 consecutive outputs n0..n0+7 (n0 a multiple of 8, so they share a tile) for token tok, CTA order.
 __device__ __forceinline__ void sum_partials8_cg(const float* __restrict__ partial, const MegaGemmShape& s, int NT, int n0,
                                                  int tok, float (&x)[8]) {
-  const int4 t = __ldg(reinterpret_cast<const int4*>(s.tiles) + (n0 >> 7));
-  const size_t slot_stride = (size_t)NT * 128;
-  const size_t off = (size_t)tok * 128 + (n0 & 127);
+  const int4 t = __ldg(reinterpret_cast<const int4*>(s.tiles) + n0 / kTileN);
+  const size_t slot_stride = (size_t)NT * kTileN;
+  const size_t off = (size_t)tok * kTileN + (n0 % kTileN);
   const float4* p = reinterpret_cast<const float4*>(partial + (size_t)t.x * slot_stride + off);
   float4 u = __ldcg(p), v = __ldcg(p + 1);
   x[0] = u.x; x[1] = u.y; x[2] = u.z; x[3] = u.w; x[4] = v.x; x[5] = v.y; x[6] = v.z; x[7] = v.w;
@@ -269,9 +277,9 @@ template <int N>
 __device__ __forceinline__ void sum_partialsN_cg(const float* __restrict__ partial, const MegaGemmShape& s, int NT, int n0,
                                                  int tok, float (&x)[N]) {
   static_assert(N == 2 || N == 4, "N");
-  const int4 t = __ldg(reinterpret_cast<const int4*>(s.tiles) + (n0 >> 7));
-  const size_t slot_stride = (size_t)NT * 128, cta_stride = slot_stride * s.max_seg;
-  const size_t off = (size_t)tok * 128 + (n0 & 127);
+  const int4 t = __ldg(reinterpret_cast<const int4*>(s.tiles) + n0 / kTileN);
+  const size_t slot_stride = (size_t)NT * kTileN, cta_stride = slot_stride * s.max_seg;
+  const size_t off = (size_t)tok * kTileN + (n0 % kTileN);
   auto add = [&](const float* p, bool first) {
     if constexpr (N == 4) {
       const float4 u = __ldcg(reinterpret_cast<const float4*>(p));
@@ -643,19 +651,19 @@ __device__ void stage_tile_argmax(const MegaArgs& a, MegaSmem* sm, int wtid) {
   uint32_t* s_key = &sm->am_key[half_id][0][0];       // [4 warps][64 batch rows]
   int* s_id = &sm->am_id[half_id][0][0];
   stage_inv_rms(a, sm, wtid);
-  const size_t slot_stride = (size_t)a.NT * 128, cta_stride = slot_stride * gs.max_seg;
+  const size_t slot_stride = (size_t)a.NT * kTileN, cta_stride = slot_stride * gs.max_seg;
   for (int tile0 = blockIdx.x * 2; tile0 < a.n_tiles_lm; tile0 += gridDim.x * 2) {
-    const int tile = tile0 + half_id;
+    const int tile = tile0 + half_id;                   // 128 vocabulary rows: one half of a 256-row GEMM tile
     const bool tile_ok = tile < a.n_tiles_lm;
     const int v = tile * 128 + t128;
     int4 ts = make_int4(0, 1, 0, 0);
-    if (tile_ok) ts = __ldg(reinterpret_cast<const int4*>(gs.tiles) + tile);
+    if (tile_ok) ts = __ldg(reinterpret_cast<const int4*>(gs.tiles) + v / kTileN);
     for (int rb = 0; rb < a.B; rb += 64) {              // 64 batch rows at a time (scratch holds 4 x 64 per half)
       const int rend = min(a.B, rb + 64);
       for (int r = rb; r < rend; ++r) {
         uint32_t key = 0;
         if (tile_ok && a.st.active[r] && v < a.V) {
-          const size_t off = (size_t)r * 128 + t128;
+          const size_t off = (size_t)r * kTileN + (v % kTileN);
           float lg = __ldcg(a.partial + (size_t)ts.x * slot_stride + off);
           for (int c = ts.y; c <= ts.z; ++c) lg += __ldcg(a.partial + (size_t)c * cta_stride + off);
           lg *= sm->inv_s[r];
@@ -735,10 +743,15 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int cta = blockIdx.x, G = gridDim.x;
   const uint32_t stage0 = (smem_u32(smem_raw) + (uint32_t)sizeof(MegaSmem) + 1023u) & ~1023u;
-  const uint32_t a_bytes = kTileM * kTileK * 2;
-  const uint32_t b_bytes = (uint32_t)a.NT * kTileK * 2;
-  const uint32_t stage_bytes = a_bytes + b_bytes;
+  // ring: S activation blocks first, then S weight blocks.  A token tile shorter than 128 rows is read
+  // by the tensor core as 128 rows anyway; the surplus rows fall on the blocks that follow.
+  const uint32_t x_tile_bytes = (uint32_t)a.x_rows * kTileK * 2;
+  const uint32_t x_bytes = (uint32_t)a.m_tiles * x_tile_bytes;
+  const uint32_t stage_tx = (uint32_t)kBlockBytes + x_bytes;
   const int S = a.stages;
+  const uint32_t x0 = stage0, w0 = stage0 + (uint32_t)S * x_bytes;
+  const int acc_bufs = a.m_tiles == 1 ? 2 : 1;       // 512 columns: two buffers of 256, or one of 2 x 256
+  constexpr uint32_t kTmemCols = 512;
   const int n_gemm = 4 * a.n_layers + 1;
 
   if (threadIdx.x == 0) {
@@ -759,7 +772,7 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
     tma_prefetch_desc(&map_act);
   }
   if (warp == 1) {
-    tmem_alloc(smem_u32(&sm->tmem_base), (uint32_t)a.tmem_cols);
+    tmem_alloc(smem_u32(&sm->tmem_base), kTmemCols);
     tmem_relinquish();
   }
   tc_fence_before();
@@ -786,8 +799,8 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
             if (!ok) break;
           }
           const uint32_t full = smem_u32(&sm->full[stage]);
-          mbar_expect_tx(full, stage_bytes);
-          bulk_load(stage0 + stage * stage_bytes, w + (size_t)it * a_bytes, a_bytes, full, hint_w);
+          mbar_expect_tx(full, stage_tx);
+          bulk_load(w0 + (uint32_t)stage * kBlockBytes, w + (size_t)it * kBlockBytes, kBlockBytes, full, hint_w);
           __threadfence_block();
           sm->w_issued = gi + 1;
         }
@@ -838,15 +851,16 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
           }
           if (!ok) break;
           const int stage = gi % S;
-          tma_load_2d(stage0 + stage * stage_bytes + a_bytes, mp, smem_u32(&sm->full[stage]), (int)(it % gs.kb) * kTileK, 0,
-                      hint_x);
+          for (int mt = 0; mt < a.m_tiles; ++mt)
+            tma_load_2d(x0 + (uint32_t)stage * x_bytes + (uint32_t)mt * x_tile_bytes, mp, smem_u32(&sm->full[stage]),
+                        (int)(it % gs.kb) * kTileK, mt * 128, hint_x);
         }
       }
     }
   } else if (warp == 1) {
     // ===================== MMA issuer =====================
     if (lane == 0) {
-      const uint32_t idesc = umma_idesc_bf16(a.NT);
+      const uint32_t idesc = umma_idesc_bf16(kTileN);     // M = 128 token lanes, N = 256 weight rows
       int gi = 0, seg = 0;
       bool ok = true;
       for (int gm = 0; gm < n_gemm && ok; ++gm) {
@@ -858,22 +872,26 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
           const int tile = (int)(it / gs.kb);
           long long seg_end = (long long)(tile + 1) * gs.kb;
           if (seg_end > it1) seg_end = it1;
-          const int buf = seg & 1;
-          ok = mega_wait(smem_u32(&sm->acc_empty[buf]), (uint32_t)(((seg >> 1) & 1) ^ 1), sm, a.status, kStatusMmaTimeout);
+          const int buf = seg % acc_bufs;
+          ok = mega_wait(smem_u32(&sm->acc_empty[buf]), (uint32_t)(((seg / acc_bufs) & 1) ^ 1), sm, a.status,
+                         kStatusMmaTimeout);
           if (!ok) break;
           tc_fence_after();
-          const uint32_t d_tmem = tmem_base + (uint32_t)(buf * a.NT);
+          const uint32_t d_tmem = tmem_base + (uint32_t)(buf * kTileN);
           bool first = true;
           for (; it < seg_end; ++it, ++gi) {
             const int stage = gi % S;
             ok = mega_wait(smem_u32(&sm->full[stage]), (uint32_t)((gi / S) & 1), sm, a.status, kStatusMmaTimeout);
             if (!ok) break;
             tc_fence_after();
-            const uint32_t sa = stage0 + stage * stage_bytes;
-            const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sa + a_bytes);
+            const uint64_t dw = smem_desc_sw128(w0 + (uint32_t)stage * kBlockBytes);
+            for (int mt = 0; mt < a.m_tiles; ++mt) {
+              const uint64_t dx = smem_desc_sw128(x0 + (uint32_t)stage * x_bytes + (uint32_t)mt * x_tile_bytes);
 #pragma unroll
-            for (int k = 0; k < kTileK / 16; ++k)
-              umma_bf16(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (first && k == 0) ? 0u : 1u);
+              for (int k = 0; k < kTileK / 16; ++k)
+                umma_bf16(d_tmem + (uint32_t)(mt * kTileN), dx + (uint64_t)(k * 2), dw + (uint64_t)(k * 2), idesc,
+                          (first && k == 0) ? 0u : 1u);
+            }
             first = false;
             umma_commit(smem_u32(&sm->empty[stage]));
           }
@@ -888,8 +906,8 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
     const int wtid = threadIdx.x - 96;
     const int wid = wtid >> 5;
     const int quarter = warp & 3;                   // tensor-memory lane quarter this warp may read
-    const int colhalf = wid >> 2;                   // warps 3-6 take the first half of the token columns
-    const int row = quarter * 32 + lane;
+    const int colhalf = wid >> 2;                   // warps 3-6 take the first 128 weight rows of a tile
+    const int acc_bufs = a.m_tiles == 1 ? 2 : 1;
     unsigned long long epoch = 0;
     int seg = 0;
     bool ok = true;
@@ -917,21 +935,29 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
         const int tile = (int)(it / gs.kb);
         long long seg_end = (long long)(tile + 1) * gs.kb;
         if (seg_end > it1) seg_end = it1;
-        const int buf = seg & 1;
-        ok = mega_wait(smem_u32(&sm->acc_full[buf]), (uint32_t)((seg >> 1) & 1), sm, a.status, kStatusEpilogueTimeout);
+        const int buf = seg % acc_bufs;
+        ok = mega_wait(smem_u32(&sm->acc_full[buf]), (uint32_t)((seg / acc_bufs) & 1), sm, a.status,
+                       kStatusEpilogueTimeout);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * a.NT);
         const size_t slot = (size_t)cta * gs.max_seg + seg_local;
-        float* dst = a.partial + slot * a.NT * 128 + row;
-        const int c0 = colhalf * (a.NT / 2), c1 = c0 + a.NT / 2;
-        for (int c = c0; c < c1; c += 8) {
-          float v[8];
-          tmem_ld8(taddr + c, v);
+        for (int mt = 0; mt < a.m_tiles; ++mt) {
+          if (mt * 128 + quarter * 32 >= a.B) continue;        // no batch row in this warp's lanes (warp-uniform)
+          const int tok = mt * 128 + quarter * 32 + lane;
+          const uint32_t taddr =
+              tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((buf + mt) * kTileN + colhalf * 128);
+          float* dst = a.partial + (slot * a.NT + tok) * kTileN + colhalf * 128;
+#pragma unroll 1
+          for (int c = 0; c < 128; c += 32) {
+            float v[32];
+            tmem_ld32(taddr + c, v);
+            if (tok < a.B) {
 #pragma unroll
-          for (int j = 0; j < 8; ++j)
-            if (c + j < a.B) dst[(size_t)(c + j) * 128] = v[j];
+              for (int j = 0; j < 32; j += 4)
+                *reinterpret_cast<float4*>(dst + c + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+            }
+          }
         }
         tc_fence_before();
         __syncwarp();
@@ -970,7 +996,7 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
   __syncthreads();
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, (uint32_t)a.tmem_cols);
+    tmem_dealloc(tmem_base, kTmemCols);
   }
 }
 

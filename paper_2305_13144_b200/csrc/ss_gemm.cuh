@@ -122,6 +122,23 @@ __device__ __forceinline__ void tmem_ld8(uint32_t taddr, float (&v)[8]) {
   v[0] = __uint_as_float(r0); v[1] = __uint_as_float(r1); v[2] = __uint_as_float(r2); v[3] = __uint_as_float(r3);
   v[4] = __uint_as_float(r4); v[5] = __uint_as_float(r5); v[6] = __uint_as_float(r6); v[7] = __uint_as_float(r7);
 }
+// 32 lanes x 32 consecutive fp32 columns.
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
 
 // Shared-memory matrix descriptor: K-major tile, 128-byte swizzle, rows of 128 bytes,
 // 8-row groups 1024 bytes apart.
@@ -239,16 +256,19 @@ gemm_wx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(hint_w));
       asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(hint_x));
       const int pre = n_it < p.stages ? n_it : p.stages;
-      // Repacked weights: iteration `it` of the (tile, k-block) space is the 16 KiB block number `it`,
-      // already in the swizzled shared-memory image, so a CTA's whole range is one contiguous span.
+      // Repacked weights: the 128-row tile `tile` at k-block `kblk` is one half of the 32 KiB block
+      // (tile / 2, kblk), already in the swizzled shared-memory image.
       const uint8_t* w_tiled = reinterpret_cast<const uint8_t*>(a.w_tiled);
+      auto w_block = [&](int tile, int kblk) {
+        return w_tiled + ((size_t)(tile >> 1) * p.kb + kblk) * (size_t)kBlockBytes + (size_t)(tile & 1) * a_bytes;
+      };
       // phase 1: weight tiles of the first ring fill, before the dependency resolves
       for (int i = 0; i < pre; ++i) {
         const long long it = it0 + i;
         const int tile = (int)(it / p.kb), kblk = (int)(it % p.kb);
         const uint32_t full = smem_u32(&hdr->full[i]);
         mbar_expect_tx(full, stage_bytes);
-        if (w_tiled) bulk_load(stage0 + i * stage_bytes, w_tiled + (size_t)it * a_bytes, a_bytes, full, hint_w);
+        if (w_tiled) bulk_load(stage0 + i * stage_bytes, w_block(tile, kblk), a_bytes, full, hint_w);
         else tma_load_2d(stage0 + i * stage_bytes, &map_w, full, kblk * kTileK, tile * kTileM, hint_w);
       }
       pdl_wait();
@@ -267,7 +287,7 @@ gemm_wx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         if (!mbar_wait(smem_u32(&hdr->empty[stage]), phase ^ 1u, a.status, kStatusProducerTimeout)) break;
         const uint32_t full = smem_u32(&hdr->full[stage]);
         mbar_expect_tx(full, stage_bytes);
-        if (w_tiled) bulk_load(stage0 + stage * stage_bytes, w_tiled + (size_t)it * a_bytes, a_bytes, full, hint_w);
+        if (w_tiled) bulk_load(stage0 + stage * stage_bytes, w_block(tile, kblk), a_bytes, full, hint_w);
         else tma_load_2d(stage0 + stage * stage_bytes, &map_w, full, kblk * kTileK, tile * kTileM, hint_w);
         tma_load_2d(stage0 + stage * stage_bytes + a_bytes, &map_x, full, kblk * kTileK, tok_tile * p.NT, hint_x);
         if (++stage == p.stages) { stage = 0; phase ^= 1u; }

@@ -21,6 +21,8 @@ int plan_first_pass(const ss_sched_cfg& c, const int32_t* prompt_len, const int3
 constexpr int kPageTokens = 32;        // tokens per key/value page
 constexpr int kTileM = 128;            // weight rows per GEMM tile (tcgen05 M)
 constexpr int kTileK = 64;             // bf16 elements per 128-byte swizzled row
+constexpr int kTileN = 256;            // weight rows per block of the tiled layout (tcgen05 N of the decode step)
+constexpr int kBlockBytes = kTileN * kTileK * 2;   // one (256-row tile, k-block) block: 32 KiB
 constexpr int kMaxBatch = 256;
 
 // Device status codes (which bounded wait expired / which check failed).
@@ -51,7 +53,7 @@ struct GemmPlan {
 
 struct GemmArgs {
   GemmPlan p;
-  const void* w_tiled; // weights repacked as contiguous 16 KiB (tile, k-block) images, or null (row-major via TMA)
+  const void* w_tiled; // weights repacked as contiguous 32 KiB (256-row tile, k-block) images, or null (row-major via TMA)
   int mode;
   int n_tok;           // valid tokens
   float* partial;      // [gridx*max_seg][NT][128]

@@ -60,9 +60,10 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
 }
 
 // ------------------------------------------------------------------------------------ weight repacking
-// Row-major [rows, K] bf16 -> the GEMM's streaming layout: 16 KiB blocks in (tile, k-block) order, each
-// the exact shared-memory image of a 128-row x 64-column tile under the 128-byte swizzle (row r at
-// r*128 bytes, its 16-byte chunk c stored at chunk position c ^ (r & 7)).  One thread per 16-byte chunk.
+// Row-major [rows, K] bf16 -> the GEMM's streaming layout: 32 KiB blocks in (tile, k-block) order, each
+// the exact shared-memory image of a 256-row x 64-column tile under the 128-byte swizzle (row r at
+// r*128 bytes, its 16-byte chunk c stored at chunk position c ^ (r & 7)).  Each half of a block is
+// the image of a 128-row tile, which is what the prompt-pass GEMM loads.  One thread per 16-byte chunk.
 // row_off places the source at a row offset of the destination matrix (q,k,v and gate,up are stacked).
 __global__ void __launch_bounds__(256)
 repack_weights_kernel(const uint4* __restrict__ src, long long rows, int K, uint8_t* __restrict__ dst, int row_off,
@@ -73,9 +74,9 @@ repack_weights_kernel(const uint4* __restrict__ src, long long rows, int K, uint
   const long long sr = id / chunks_per_row;
   const int cc = (int)(id - sr * chunks_per_row);
   const long long n = row_off + sr;
-  const long long tile = n >> 7;
-  const int r = (int)(n & 127), k = cc >> 3, c = cc & 7;
-  uint8_t* blk = dst + ((size_t)tile * kb + k) * (size_t)(kTileM * kTileK * 2);
+  const long long tile = n / kTileN;
+  const int r = (int)(n % kTileN), k = cc >> 3, c = cc & 7;
+  uint8_t* blk = dst + ((size_t)tile * kb + k) * (size_t)kBlockBytes;
   *reinterpret_cast<uint4*>(blk + r * 128 + ((c ^ (r & 7)) << 4)) = src[id];
 }
 

@@ -32,7 +32,23 @@ struct LayerWeights {
 };
 
 inline size_t tiled_bytes(int64_t n_out, int64_t K) {
-  return (size_t)ceil_div((int)n_out, kTileM) * ceil_div((int)K, kTileK) * (size_t)(kTileM * kTileK * 2);
+  return (size_t)ceil_div((int)n_out, kTileN) * ceil_div((int)K, kTileK) * (size_t)kBlockBytes;
+}
+
+// Split of a decode projection: 256-row tiles x k-blocks in equal contiguous ranges over the CTAs.
+struct DecodeSplit {
+  int n_tiles, kb, gsplit, max_seg;
+  long long total;
+};
+DecodeSplit plan_decode(int n_out, int K, int n_sm) {
+  DecodeSplit p{};
+  p.n_tiles = ceil_div(n_out, kTileN);
+  p.kb = ceil_div(K, kTileK);
+  p.total = (long long)p.n_tiles * p.kb;
+  p.gsplit = (int)std::min<long long>(n_sm, p.total);
+  const int ipc = std::max(1, (int)((p.total + p.gsplit - 1) / p.gsplit));
+  p.max_seg = (ipc + p.kb - 2) / p.kb + 1;
+  return p;
 }
 
 GemmPlan plan_gemm(int n_out, int K, int NT, int tok_tiles, int mode, int n_sm) {
@@ -86,6 +102,22 @@ std::vector<TileSeg> tile_table(const GemmPlan& p) {
   return t;
 }
 
+std::vector<TileSeg> decode_tile_table(const DecodeSplit& p) {
+  SplitInfo s{};
+  s.gridx = p.gsplit;
+  s.kb = p.kb;
+  s.max_seg = p.max_seg;
+  s.total = p.total;
+  std::vector<TileSeg> t(p.n_tiles);
+  for (int tile = 0; tile < p.n_tiles; ++tile) {
+    const long long x0 = (long long)tile * p.kb;
+    const int c0 = split_owner(s, x0), c1 = split_owner(s, x0 + p.kb - 1);
+    const int seg0 = tile - (int)(split_begin(s, c0) / p.kb);
+    t[tile] = {c0 * p.max_seg + seg0, c0 + 1, c1, 0};
+  }
+  return t;
+}
+
 }  // namespace
 
 struct ss_ctx {
@@ -124,7 +156,8 @@ struct ss_ctx {
   bf16 *x_dec = nullptr, *o_dec = nullptr, *act_dec = nullptr;
   float* partial = nullptr;
   size_t partial_bytes = 0;
-  TileSeg* tbl[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};   // qkv, o, gate/up, down, lm head
+  TileSeg* tbl[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};   // decode step: qkv, o, gate/up, down, lm head
+  TileSeg* tbl_lm_prompt = nullptr;                                  // LM head after the prompt pass (128-row tiles)
   float* rowss = nullptr;          // [kMaxBatch][kMaxSlices]
   unsigned long long* grid_ctr = nullptr;
   unsigned long long* trace = nullptr;  // stage-boundary time stamps of the last decode step
@@ -253,7 +286,7 @@ struct Offsets {
   std::vector<size_t> attn_norm, wqkv, wo, ffn_norm, wgu, wdown;
   size_t inv_freq, status, rows, block_table, out_tokens, tok, h, x, qkv, attn_o, gu, act;
   size_t h_dec, x_dec, o_dec, act_dec, partial, kv;
-  size_t tbl[5], tile_val, tile_idx, rowss, grid_ctr, wptr, norm_ptr, trace;
+  size_t tbl[5], tbl_lm_prompt, tile_val, tile_idx, rowss, grid_ctr, wptr, norm_ptr, trace;
   size_t partial_bytes;
   int R, max_pages, n_pages;
   size_t total;
@@ -313,7 +346,11 @@ void layout(const ss_model_cfg& m, const ss_runtime_cfg& rt, int n_sm, Offsets& 
   size_t pb = 0;
   const int shapes[5][2] = {{(int)(3 * d), (int)d}, {(int)d, (int)d}, {(int)(2 * F), (int)d}, {(int)d, (int)F}, {(int)V, (int)d}};
   for (auto& s : shapes) {
-    GemmPlan p = plan_gemm(s[0], s[1], NTmax, 1, kGemmPartial, n_sm);
+    const DecodeSplit p = plan_decode(s[0], s[1], n_sm);
+    pb = std::max(pb, (size_t)p.gsplit * p.max_seg * NTmax * kTileN * sizeof(float));
+  }
+  {
+    const GemmPlan p = plan_gemm((int)V, (int)d, NTmax, 1, kGemmPartial, n_sm);
     pb = std::max(pb, (size_t)p.gridx * p.max_seg * p.NT * 128 * sizeof(float));
   }
   o.partial_bytes = pb;
@@ -323,7 +360,8 @@ void layout(const ss_model_cfg& m, const ss_runtime_cfg& rt, int n_sm, Offsets& 
   o.wptr = a.take((size_t)(4 * m.n_layers + 1) * sizeof(void*));
   o.norm_ptr = a.take((size_t)(2 * m.n_layers + 1) * sizeof(void*));
   o.trace = a.take((size_t)(2 + 4 * (4 * m.n_layers + 1)) * 8);
-  for (int i = 0; i < 5; ++i) o.tbl[i] = a.take((size_t)ceil_div(shapes[i][0], kTileM) * sizeof(TileSeg));
+  for (int i = 0; i < 5; ++i) o.tbl[i] = a.take((size_t)ceil_div(shapes[i][0], kTileN) * sizeof(TileSeg));
+  o.tbl_lm_prompt = a.take((size_t)ceil_div((int)V, kTileM) * sizeof(TileSeg));
   o.tile_val = a.take((size_t)kMaxBatch * ceil_div((int)V, kTileM) * 4);
   o.tile_idx = a.take((size_t)kMaxBatch * ceil_div((int)V, kTileM) * 4);
   o.n_pages = (int)((rt.kv_pool_tokens + kPageTokens - 1) / kPageTokens) + rt.max_batch;
@@ -391,7 +429,8 @@ int enqueue_decode_step(ss_ctx* c, const ss_step_opts* opts, int32_t* next_token
   const int NT = round_up(B, 16);
   const CUtensorMap *mx, *mo, *ma;
   int rc;
-  if ((rc = xmap(c, 3, NT, &mx)) || (rc = xmap(c, 4, NT, &mo)) || (rc = xmap(c, 5, NT, &ma))) return rc;
+  const int xr = NT > 128 ? 128 : NT;          // activation rows per TMA load
+  if ((rc = xmap(c, 3, xr, &mx)) || (rc = xmap(c, 4, xr, &mo)) || (rc = xmap(c, 5, xr, &ma))) return rc;
   MegaArgs a{};
   a.n_layers = m.n_layers; a.d = d; a.H = m.n_heads; a.Dh = m.head_dim; a.F = F; a.V = V; a.eos_id = m.eos_id;
   a.eps = m.rms_eps;
@@ -402,19 +441,18 @@ int enqueue_decode_step(ss_ctx* c, const ss_step_opts* opts, int32_t* next_token
   const int shp[5][2] = {{3 * d, d}, {d, d}, {2 * F, d}, {d, F}, {V, d}};
   size_t need_partial = 0;
   for (int i = 0; i < 5; ++i) {
-    const GemmPlan p = plan_gemm(shp[i][0], shp[i][1], NT, 1, kGemmPartial, c->n_sm);
-    a.shape[i] = {p.n_tiles, p.kb, p.max_seg, p.gridx, (long long)p.n_tiles * p.kb, c->tbl[i]};
-    need_partial = std::max(need_partial, (size_t)p.gridx * p.max_seg * NT * 128 * sizeof(float));
+    const DecodeSplit p = plan_decode(shp[i][0], shp[i][1], c->n_sm);
+    a.shape[i] = {p.n_tiles, p.kb, p.max_seg, p.gsplit, p.total, c->tbl[i]};
+    need_partial = std::max(need_partial, (size_t)p.gsplit * p.max_seg * NT * kTileN * sizeof(float));
   }
   if (need_partial > c->partial_bytes) return SS_ERR_CAPACITY;
   a.B = B; a.NT = NT;
-  const int stage_bytes = kTileM * kTileK * 2 + NT * kTileK * 2;
+  a.m_tiles = NT > 128 ? 2 : 1;
+  a.x_rows = NT > 128 ? 128 : NT;
+  const int stage_bytes = kBlockBytes + a.m_tiles * a.x_rows * kTileK * 2;
   const int header = (int)sizeof(MegaSmem) + 1024;
   a.stages = std::max(2, std::min(kGemmMaxStages, (227 * 1024 - header) / stage_bytes));
   const size_t smem = (size_t)header + (size_t)a.stages * stage_bytes;
-  int cols = 32;
-  while (cols < 2 * NT) cols <<= 1;
-  a.tmem_cols = cols;
   a.st = c->st; a.kv = c->kv;
   a.h = c->h_dec; a.x = c->x_dec; a.o = c->o_dec; a.act = c->act_dec;
   a.rowss = c->rowss; a.partial = c->partial;
@@ -614,10 +652,14 @@ int ss_create(const ss_model_cfg* model, const ss_runtime_cfg* rt, void* dev_are
     const int shp[5][2] = {{(int)(3 * d), (int)d}, {(int)d, (int)d}, {(int)(2 * F), (int)d}, {(int)d, (int)F}, {(int)V, (int)d}};
     for (int i = 0; i < 5; ++i) {
       c->tbl[i] = (TileSeg*)(A + o.tbl[i]);
-      const std::vector<TileSeg> t = tile_table(plan_gemm(shp[i][0], shp[i][1], 16, 1, kGemmPartial, c->n_sm));
+      const std::vector<TileSeg> t = decode_tile_table(plan_decode(shp[i][0], shp[i][1], c->n_sm));
       if (cudaMemcpy(c->tbl[i], t.data(), t.size() * sizeof(TileSeg), cudaMemcpyHostToDevice) != cudaSuccess)
         return fail(SS_ERR_CUDA);
     }
+    c->tbl_lm_prompt = (TileSeg*)(A + o.tbl_lm_prompt);
+    const std::vector<TileSeg> t = tile_table(plan_gemm((int)V, (int)d, 16, 1, kGemmPartial, c->n_sm));
+    if (cudaMemcpy(c->tbl_lm_prompt, t.data(), t.size() * sizeof(TileSeg), cudaMemcpyHostToDevice) != cudaSuccess)
+      return fail(SS_ERR_CUDA);
   }
   c->kv.pool = (bf16*)(A + o.kv);
   c->kv.page_elems = (size_t)2 * model->n_heads * kPageTokens * model->head_dim;
@@ -799,7 +841,7 @@ int ss_prefill(ss_ctx* c, const int32_t* tokens, const int32_t* cu, int32_t B, c
   const GemmPlan p_lm = plan_gemm(m.vocab, m.d_model, NT, 1, kGemmPartial, c->n_sm);
   if ((rc = run_gemm(c, c->lm_head, *mx, p_lm, kGemmPartial, B, nullptr, nullptr, 0))) return bail(rc);
   SS_CUDA_B(launch(c, lmhead_tile_argmax_kernel, dim3(c->n_tiles_lm), dim3(128), 0, (const float*)c->partial,
-                   split_of(p_lm, c->tbl[4]), c->st, opts ? opts->dump_logits : (float*)nullptr, c->tile_val,
+                   split_of(p_lm, c->tbl_lm_prompt), c->st, opts ? opts->dump_logits : (float*)nullptr, c->tile_val,
                    c->tile_idx, B, m.vocab, c->n_tiles_lm, m.eos_id));
   SS_CUDA_B(launch(c, bookkeeping_kernel, dim3(1), dim3(1024), 0, c->st, (const float*)c->tile_val,
                    (const int32_t*)c->tile_idx, c->n_tiles_lm, opts ? opts->forced_tokens : (const int32_t*)nullptr,
