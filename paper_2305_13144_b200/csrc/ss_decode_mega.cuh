@@ -36,8 +36,8 @@ namespace ss {
 
 constexpr int kMegaThreads = 352;
 constexpr int kMegaWorkers = 256;          // warps 3..10
-constexpr int kRowSlice = 512;             // elements of a row handled by one residual work item
-constexpr int kMaxSlices = 16;             // d_model <= 8192
+constexpr int kRowSlice = 128;             // elements of a row handled by one residual work item (one warp, 4 per lane)
+constexpr int kMaxSlices = 64;             // d_model <= 8192
 
 enum : uint32_t { kStatusGridBarrierTimeout = 5, kStatusFlagTimeout = 6 };
 
@@ -170,90 +170,132 @@ __device__ __forceinline__ bool grid_barrier(const MegaArgs& a, MegaSmem* sm, un
   return sm->abort == 0;
 }
 
-// Sum of the partials of output row n for token tok (CTA order), read past L1.
-__device__ __forceinline__ float sum_partials_cg(const float* __restrict__ partial, const MegaGemmShape& s, int NT, int n, int tok) {
-  const int4 t = __ldg(reinterpret_cast<const int4*>(s.tiles) + n / kTileN);
-  const size_t slot_stride = (size_t)NT * kTileN;
-  const size_t off = (size_t)tok * kTileN + (n % kTileN);
-  float acc = __ldcg(partial + (size_t)t.x * slot_stride + off);
-  const size_t cta_stride = slot_stride * s.max_seg;
-  for (int c = t.y; c <= t.z; ++c) acc += __ldcg(partial + (size_t)c * cta_stride + off);
-  return acc;
+// The stages between projections are chains of dependent L2 round trips (~0.7 us each), not bandwidth: the
+// helpers below put independent loads in flight together and keep only true dependencies serial.
+
+template <int N>
+__device__ __forceinline__ void ldcg_vec(const float* p, float (&x)[N]) {
+  static_assert(N == 2 || N == 4 || N == 8, "N");
+  if constexpr (N == 2) {
+    const float2 u = __ldcg(reinterpret_cast<const float2*>(p));
+    x[0] = u.x; x[1] = u.y;
+  } else {
+#pragma unroll
+    for (int i = 0; i < N; i += 4) {
+      const float4 u = __ldcg(reinterpret_cast<const float4*>(p + i));
+      x[i] = u.x; x[i + 1] = u.y; x[i + 2] = u.z; x[i + 3] = u.w;
+    }
+  }
 }
 
-__device__ __forceinline__ float row_inv_rms(const MegaArgs& a, int r) {
+// Sum of the partials of the N consecutive outputs n0.. (inside one tile) for token tok, read past L1: the
+// tile's first segment, then segment 0 of CTAs c_next..c_last.  Up to BATCH segment loads are in flight
+// together; the additions stay in CTA order, so the sum does not depend on timing.
+template <int N, int BATCH>
+__device__ __forceinline__ void sum_partials_cg(const float* __restrict__ partial, const MegaGemmShape& s, int NT, int n0,
+                                                int tok, float (&x)[N]) {
+  const int4 t = __ldg(reinterpret_cast<const int4*>(s.tiles) + n0 / kTileN);
+  const size_t slot_stride = (size_t)NT * kTileN, cta_stride = slot_stride * s.max_seg;
+  const size_t off = (size_t)tok * kTileN + (n0 % kTileN);
+  ldcg_vec<N>(partial + (size_t)t.x * slot_stride + off, x);
+  for (int c = t.y; c <= t.z; c += BATCH) {
+    float u[BATCH][N];
+#pragma unroll
+    for (int j = 0; j < BATCH; ++j)        // past the last segment: re-read the last one (dropped below)
+      ldcg_vec<N>(partial + (size_t)min(c + j, t.z) * cta_stride + off, u[j]);
+#pragma unroll
+    for (int j = 0; j < BATCH; ++j) {
+      const bool on = c + j <= t.z;
+#pragma unroll
+      for (int i = 0; i < N; ++i) x[i] += on ? u[j][i] : 0.f;
+    }
+  }
+}
+
+// 1/rms of row r; warp-collective (every lane returns it).  Lane i reads slices i, i+32.
+__device__ __forceinline__ float warp_row_inv_rms(const MegaArgs& a, int r, int lane) {
   const int ns = (a.d + kRowSlice - 1) / kRowSlice;
   float ss = 0.f;
-  for (int s = 0; s < ns; ++s) ss += __ldcg(a.rowss + (size_t)r * kMaxSlices + s);
+  for (int i = lane; i < ns; i += 32) ss += __ldcg(a.rowss + (size_t)r * kMaxSlices + i);
+  ss = warp_sum(ss);
   return rsqrtf(ss / a.d + a.eps);
 }
 
 // ---- stage: embedding (or residual add) + lazy RMSNorm operand -------------------------------------
-// Work item = (row, slice of kRowSlice elements), dealt to CTAs; 256 worker threads, 2 elements each.
+// Work unit = (row, slice of 128 columns) per warp, 4 columns per lane; units are dealt round-robin over
+// the CTAs first, so the whole stage is one pass with a few warps busy in every CTA.
 // mode 0: h = E[cur_tok]; mode 1: h += projection (partials of shape `gs`).
-__device__ void stage_residual(const MegaArgs& a, MegaSmem* sm, int wtid, int mode, const MegaGemmShape* gs,
+__device__ void stage_residual(const MegaArgs& a, int wtid, int mode, const MegaGemmShape* gs,
                                const bf16* __restrict__ gain, bool dump) {
   const int ns = (a.d + kRowSlice - 1) / kRowSlice;
-  const int n_items = a.B * ns;
+  const int n_units = a.B * ns;
   const int lane = wtid & 31, wid = wtid >> 5;
-  for (int item = blockIdx.x; item < n_items; item += gridDim.x) {
-    const int r = item / ns, sl = item - r * ns;
+  for (int u = wid * gridDim.x + blockIdx.x; u < n_units; u += 8 * gridDim.x) {
+    const int r = u / ns, sl = u - r * ns;
+    if (!a.st.active[r]) continue;
+    const int c = sl * kRowSlice + lane * 4;
     float ss = 0.f;
-    if (a.st.active[r]) {
-      int tok = 0;
+    if (c < a.d) {
+      float v[4];
       if (mode == 0) {
-        tok = a.st.cur_tok[r];
+        int tok = a.st.cur_tok[r];
         if (tok < 0 || tok >= a.V) tok = 0;
+        const uint2 e = __ldg(reinterpret_cast<const uint2*>(a.embed + (size_t)tok * a.d + c));
+        const float2 e0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&e.x));
+        const float2 e1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&e.y));
+        v[0] = e0.x; v[1] = e0.y; v[2] = e1.x; v[3] = e1.y;
+      } else {
+        const float4 h4 = __ldcg(reinterpret_cast<const float4*>(a.h + (size_t)r * a.d + c));
+        sum_partials_cg<4, 12>(a.partial, *gs, a.NT, c, r, v);
+        v[0] += h4.x; v[1] += h4.y; v[2] += h4.z; v[3] += h4.w;
       }
-#pragma unroll
-      for (int j = 0; j < kRowSlice / kMegaWorkers; ++j) {
-        const int i = sl * kRowSlice + wtid + j * kMegaWorkers;
-        if (i < a.d) {
-          float v;
-          if (mode == 0) v = __bfloat162float(a.embed[(size_t)tok * a.d + i]);
-          else v = __ldcg(a.h + (size_t)r * a.d + i) + sum_partials_cg(a.partial, *gs, a.NT, i, r);
-          a.h[(size_t)r * a.d + i] = v;
-          if (dump && a.dump_hidden) a.dump_hidden[(size_t)r * a.d + i] = v;
-          a.x[(size_t)r * a.d + i] = __float2bfloat16_rn(v * __bfloat162float(gain[i]));
-          ss += v * v;
-        }
-      }
+      const uint2 gb = __ldg(reinterpret_cast<const uint2*>(gain + c));
+      const float2 g0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gb.x));
+      const float2 g1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&gb.y));
+      *reinterpret_cast<float4*>(a.h + (size_t)r * a.d + c) = make_float4(v[0], v[1], v[2], v[3]);
+      if (dump && a.dump_hidden)
+        *reinterpret_cast<float4*>(a.dump_hidden + (size_t)r * a.d + c) = make_float4(v[0], v[1], v[2], v[3]);
+      __align__(8) bf16 xb[4];
+      xb[0] = __float2bfloat16_rn(v[0] * g0.x); xb[1] = __float2bfloat16_rn(v[1] * g0.y);
+      xb[2] = __float2bfloat16_rn(v[2] * g1.x); xb[3] = __float2bfloat16_rn(v[3] * g1.y);
+      *reinterpret_cast<uint2*>(a.x + (size_t)r * a.d + c) = *reinterpret_cast<const uint2*>(xb);
+      ss = v[0] * v[0] + v[1] * v[1] + v[2] * v[2] + v[3] * v[3];
     }
     ss = warp_sum(ss);
-    named_bar_workers();
-    if (lane == 0) sm->red[wid] = ss;
-    named_bar_workers();
-    if (wtid == 0 && a.st.active[r]) {
-      float t = 0.f;
-#pragma unroll
-      for (int w = 0; w < 8; ++w) t += sm->red[w];
-      a.rowss[(size_t)r * kMaxSlices + sl] = t;
-    }
+    if (lane == 0) a.rowss[(size_t)r * kMaxSlices + sl] = ss;
   }
 }
 
 // ---- helpers shared by the stages ----------------------------------------------------------------------
-// 8 consecutive outputs n0..n0+7 (n0 a multiple of 8, so they share a tile) for token tok, CTA order.
-__device__ __forceinline__ void sum_partials8_cg(const float* __restrict__ partial, const MegaGemmShape& s, int NT, int n0,
-                                                 int tok, float (&x)[8]) {
-  const int4 t = __ldg(reinterpret_cast<const int4*>(s.tiles) + n0 / kTileN);
-  const size_t slot_stride = (size_t)NT * kTileN;
-  const size_t off = (size_t)tok * kTileN + (n0 % kTileN);
-  const float4* p = reinterpret_cast<const float4*>(partial + (size_t)t.x * slot_stride + off);
-  float4 u = __ldcg(p), v = __ldcg(p + 1);
-  x[0] = u.x; x[1] = u.y; x[2] = u.z; x[3] = u.w; x[4] = v.x; x[5] = v.y; x[6] = v.z; x[7] = v.w;
-  const size_t cta_stride = slot_stride * s.max_seg;
-  for (int c = t.y; c <= t.z; ++c) {
-    p = reinterpret_cast<const float4*>(partial + (size_t)c * cta_stride + off);
-    u = __ldcg(p);
-    v = __ldcg(p + 1);
-    x[0] += u.x; x[1] += u.y; x[2] += u.z; x[3] += u.w; x[4] += v.x; x[5] += v.y; x[6] += v.z; x[7] += v.w;
+// 1/rms of every active row into shared memory: warp w takes rows w, w+8, ... (four rows' loads in flight).
+// Split in two so that a stage can put its own loads in flight between the halves.
+struct InvRmsLoads { float s[4]; };
+__device__ __forceinline__ InvRmsLoads inv_rms_issue(const MegaArgs& a, int r0, int lane) {
+  const int ns = (a.d + kRowSlice - 1) / kRowSlice;
+  InvRmsLoads q;
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const int r = r0 + 8 * k;
+    q.s[k] = 0.f;
+    if (r < a.B && a.st.active[r])
+      for (int i = lane; i < ns; i += 32) q.s[k] += __ldcg(a.rowss + (size_t)r * kMaxSlices + i);
+  }
+  return q;
+}
+__device__ __forceinline__ void inv_rms_finish(const MegaArgs& a, MegaSmem* sm, const InvRmsLoads& q, int r0, int lane) {
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    const int r = r0 + 8 * k;
+    const float t = warp_sum(q.s[k]);
+    if (r < a.B && lane == 0) sm->inv_s[r] = a.st.active[r] ? rsqrtf(t / a.d + a.eps) : 0.f;
   }
 }
-
-// 1/rms of every active row into shared memory (one pass at the start of a consumer stage).
 __device__ __forceinline__ void stage_inv_rms(const MegaArgs& a, MegaSmem* sm, int wtid) {
-  for (int r = wtid; r < a.B; r += kMegaWorkers) sm->inv_s[r] = a.st.active[r] ? row_inv_rms(a, r) : 0.f;
+  const int lane = wtid & 31, wid = wtid >> 5;
+  for (int r0 = wid; r0 < a.B; r0 += 32) {
+    const InvRmsLoads q = inv_rms_issue(a, r0, lane);
+    inv_rms_finish(a, sm, q, r0, lane);
+  }
   named_bar_workers();
 }
 
@@ -273,28 +315,6 @@ __device__ __forceinline__ void group_bar(int id, int threads) {
 // Scan layout: a key row is Dh/8 chunks of 16 bytes; lane (g, gl) of the warp handles key g of the
 // load step and chunks gl, gl+GROUP, gl+2*GROUP, gl+3*GROUP, so each warp-wide load reads 64
 // contiguous bytes per key (full sectors).
-template <int N>
-__device__ __forceinline__ void sum_partialsN_cg(const float* __restrict__ partial, const MegaGemmShape& s, int NT, int n0,
-                                                 int tok, float (&x)[N]) {
-  static_assert(N == 2 || N == 4, "N");
-  const int4 t = __ldg(reinterpret_cast<const int4*>(s.tiles) + n0 / kTileN);
-  const size_t slot_stride = (size_t)NT * kTileN, cta_stride = slot_stride * s.max_seg;
-  const size_t off = (size_t)tok * kTileN + (n0 % kTileN);
-  auto add = [&](const float* p, bool first) {
-    if constexpr (N == 4) {
-      const float4 u = __ldcg(reinterpret_cast<const float4*>(p));
-      if (first) { x[0] = u.x; x[1] = u.y; x[2] = u.z; x[3] = u.w; }
-      else { x[0] += u.x; x[1] += u.y; x[2] += u.z; x[3] += u.w; }
-    } else {
-      const float2 u = __ldcg(reinterpret_cast<const float2*>(p));
-      if (first) { x[0] = u.x; x[1] = u.y; }
-      else { x[0] += u.x; x[1] += u.y; }
-    }
-  };
-  add(partial + (size_t)t.x * slot_stride + off, true);
-  for (int c = t.y; c <= t.z; ++c) add(partial + (size_t)c * cta_stride + off, false);
-}
-
 constexpr int kAttnPass = 8;               // pairs per pass (= worker warps)
 constexpr int kAttnSlots = 9;              // partials per pair: one per warp + the new token
 
@@ -441,7 +461,7 @@ __device__ void stage_attention(const MegaArgs& a, MegaSmem* sm, int wtid, int l
       const int p = sm->pair_id[wid];
       const int r = p / H, hd = p - r * H;
       const int pos = single ? sm->pair_pos[wid] : a.st.ctx_len[r];
-      const float inv = row_inv_rms(a, r);
+      const float inv = warp_row_inv_rms(a, r, lane);
       const int e0 = lane * EPL;
       float sn[EPL], cs[EPL];
 #pragma unroll
@@ -450,9 +470,9 @@ __device__ void stage_attention(const MegaArgs& a, MegaSmem* sm, int wtid, int l
         else sincosf((float)pos * a.inv_freq[(lane & 15) * EPL + j], &sn[j], &cs[j]);
       }
       float qx[EPL], kx[EPL], vx[EPL];
-      sum_partialsN_cg<EPL>(a.partial, gs, a.NT, hd * DH + e0, r, qx);
-      sum_partialsN_cg<EPL>(a.partial, gs, a.NT, d + hd * DH + e0, r, kx);
-      sum_partialsN_cg<EPL>(a.partial, gs, a.NT, 2 * d + hd * DH + e0, r, vx);
+      sum_partials_cg<EPL, 4>(a.partial, gs, a.NT, hd * DH + e0, r, qx);
+      sum_partials_cg<EPL, 4>(a.partial, gs, a.NT, d + hd * DH + e0, r, kx);
+      sum_partials_cg<EPL, 4>(a.partial, gs, a.NT, 2 * d + hd * DH + e0, r, vx);
       int pg = single ? sm->pair_pgnew[wid] : a.st.block_table[(size_t)r * a.st.max_pages + pos / kPageTokens];
       if (pg < 0 || pg >= a.kv.n_pages) { atomicCAS(a.status, 0u, (uint32_t)kStatusBadPage); pg = -1; }
       bf16* kdst = a.kv.pool + (size_t)layer * a.kv.layer_stride + (size_t)(pg < 0 ? 0 : pg) * a.kv.page_elems +
@@ -620,26 +640,53 @@ __device__ void stage_attention(const MegaArgs& a, MegaSmem* sm, int wtid, int l
 }
 
 // ---- stage: SwiGLU ----------------------------------------------------------------------------------
-// 8 consecutive features per thread (two 128-bit loads per partial segment, one 128-bit store).
+// 8 consecutive features per thread (two 128-bit loads per partial segment, one 128-bit store).  The loads
+// for 1/rms and the first unit's partials are in flight together.
 __device__ void stage_swiglu(const MegaArgs& a, MegaSmem* sm, int wtid) {
   const MegaGemmShape& gs = a.shape[2];
-  stage_inv_rms(a, sm, wtid);
+  const int lane = wtid & 31, wid = wtid >> 5;
   const int F8 = a.F >> 3;
-  const long long n = (long long)a.B * F8;
-  for (long long e = (long long)blockIdx.x * kMegaWorkers + wtid; e < n; e += (long long)gridDim.x * kMegaWorkers) {
-    const int r = (int)(e / F8), f0 = (int)(e - (long long)r * F8) << 3;
-    if (!a.st.active[r]) continue;
-    const float inv = sm->inv_s[r];
-    float gt[8], up[8];
-    sum_partials8_cg(a.partial, gs, a.NT, f0, r, gt);
-    sum_partials8_cg(a.partial, gs, a.NT, a.F + f0, r, up);
-    __align__(16) bf16 ob[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-      const float gv = gt[j] * inv;
-      ob[j] = __float2bfloat16_rn(gv / (1.f + __expf(-gv)) * (up[j] * inv));
+  const long long n = (long long)a.B * F8, stride = (long long)gridDim.x * kMegaWorkers;
+  long long e = (long long)blockIdx.x * kMegaWorkers + wtid;
+  const InvRmsLoads q = inv_rms_issue(a, wid, lane);
+  float gt[8], up[8];
+  int r = 0, f0 = 0;
+  bool have = false;
+  if (e < n) {
+    r = (int)(e / F8);
+    f0 = (int)(e - (long long)r * F8) << 3;
+    have = a.st.active[r] != 0;
+    if (have) {
+      sum_partials_cg<8, 2>(a.partial, gs, a.NT, f0, r, gt);
+      sum_partials_cg<8, 2>(a.partial, gs, a.NT, a.F + f0, r, up);
     }
-    *reinterpret_cast<uint4*>(a.act + (size_t)r * a.F + f0) = *reinterpret_cast<const uint4*>(ob);
+  }
+  inv_rms_finish(a, sm, q, wid, lane);
+  for (int r0 = wid + 32; r0 < a.B; r0 += 32) {
+    const InvRmsLoads q2 = inv_rms_issue(a, r0, lane);
+    inv_rms_finish(a, sm, q2, r0, lane);
+  }
+  named_bar_workers();
+  for (;;) {
+    if (have) {
+      const float inv = sm->inv_s[r];
+      __align__(16) bf16 ob[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const float gv = gt[j] * inv;
+        ob[j] = __float2bfloat16_rn(gv / (1.f + __expf(-gv)) * (up[j] * inv));
+      }
+      *reinterpret_cast<uint4*>(a.act + (size_t)r * a.F + f0) = *reinterpret_cast<const uint4*>(ob);
+    }
+    e += stride;
+    if (e >= n) break;
+    r = (int)(e / F8);
+    f0 = (int)(e - (long long)r * F8) << 3;
+    have = a.st.active[r] != 0;
+    if (have) {
+      sum_partials_cg<8, 2>(a.partial, gs, a.NT, f0, r, gt);
+      sum_partials_cg<8, 2>(a.partial, gs, a.NT, a.F + f0, r, up);
+    }
   }
 }
 
@@ -917,7 +964,7 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
     if (tracer) a.trace[tr++] = global_timer_ns();
     if (cta == 0 && wtid == 0) a.st.scalars[1] = 0;   // rows still active after this step (counted in the last stage)
     attention_setup<DH>(a, sm, wtid);
-    stage_residual(a, sm, wtid, 0, nullptr, a.norm_ptr[0], a.n_layers == 0);
+    stage_residual(a, wtid, 0, nullptr, a.norm_ptr[0], a.n_layers == 0);
     ok = grid_barrier(a, sm, epoch, wtid);
     if (ok && wtid == 0) sm->act_epoch = 1;
     if (tracer) a.trace[tr++] = global_timer_ns();
@@ -975,11 +1022,11 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
       if (type == 0) {
         stage_attention<DH>(a, sm, wtid, layer);
       } else if (type == 1) {
-        stage_residual(a, sm, wtid, 1, &a.shape[1], a.norm_ptr[2 * layer + 1], false);
+        stage_residual(a, wtid, 1, &a.shape[1], a.norm_ptr[2 * layer + 1], false);
       } else if (type == 2) {
         stage_swiglu(a, sm, wtid);
       } else if (type == 3) {
-        stage_residual(a, sm, wtid, 1, &a.shape[3], a.norm_ptr[2 * layer + 2], layer + 1 == a.n_layers);
+        stage_residual(a, wtid, 1, &a.shape[3], a.norm_ptr[2 * layer + 2], layer + 1 == a.n_layers);
       } else {
         stage_tile_argmax(a, sm, wtid);
       }
