@@ -188,21 +188,48 @@ __device__ __forceinline__ void ldcg_vec(const float* p, float (&x)[N]) {
   }
 }
 
-// Sum of the partials of the N consecutive outputs n0.. (inside one tile) for token tok, read past L1: the
-// tile's first segment, then segment 0 of CTAs c_next..c_last.  Up to BATCH segment loads are in flight
-// together; the additions stay in CTA order, so the sum does not depend on timing.
+// Partial sums of the N consecutive outputs n0.. (inside one tile) for token tok, read past L1: the tile's
+// first segment, then segment 0 of CTAs c_next..c_last (additions in CTA order, so the sum does not depend
+// on timing).  Split in three so that a stage can put the loads of several sums in flight before it waits:
+//   tile_seg()       the tile's table entry (one load);
+//   partials_issue() the first segment and the next BATCH segments (loads only, unconditional so that they
+//                    stay in registers: past the last segment the last one is read again and dropped);
+//   partials_sum()   the additions, and any segments beyond the first batch.
+__device__ __forceinline__ int4 tile_seg(const MegaGemmShape& s, int n0) {
+  return __ldg(reinterpret_cast<const int4*>(s.tiles) + n0 / kTileN);
+}
 template <int N, int BATCH>
-__device__ __forceinline__ void sum_partials_cg(const float* __restrict__ partial, const MegaGemmShape& s, int NT, int n0,
-                                                int tok, float (&x)[N]) {
-  const int4 t = __ldg(reinterpret_cast<const int4*>(s.tiles) + n0 / kTileN);
+struct PartialLoads {
+  float x[N];
+  float u[BATCH][N];
+};
+template <int N, int BATCH>
+__device__ __forceinline__ void partials_issue(const float* __restrict__ partial, const MegaGemmShape& s, int NT, const int4 t,
+                                               int n0, int tok, PartialLoads<N, BATCH>& q) {
   const size_t slot_stride = (size_t)NT * kTileN, cta_stride = slot_stride * s.max_seg;
   const size_t off = (size_t)tok * kTileN + (n0 % kTileN);
-  ldcg_vec<N>(partial + (size_t)t.x * slot_stride + off, x);
-  for (int c = t.y; c <= t.z; c += BATCH) {
+  ldcg_vec<N>(partial + (size_t)t.x * slot_stride + off, q.x);
+#pragma unroll
+  for (int j = 0; j < BATCH; ++j) ldcg_vec<N>(partial + (size_t)min(t.y + j, t.z) * cta_stride + off, q.u[j]);
+}
+template <int N, int BATCH>
+__device__ __forceinline__ void partials_sum(const float* __restrict__ partial, const MegaGemmShape& s, int NT, const int4 t,
+                                             int n0, int tok, const PartialLoads<N, BATCH>& q, float (&x)[N]) {
+#pragma unroll
+  for (int i = 0; i < N; ++i) x[i] = q.x[i];
+  if (t.y > t.z) return;
+#pragma unroll
+  for (int j = 0; j < BATCH; ++j) {
+    const bool on = t.y + j <= t.z;
+#pragma unroll
+    for (int i = 0; i < N; ++i) x[i] += on ? q.u[j][i] : 0.f;
+  }
+  const size_t cta_stride = (size_t)NT * kTileN * s.max_seg;
+  const size_t off = (size_t)tok * kTileN + (n0 % kTileN);
+  for (int c = t.y + BATCH; c <= t.z; c += BATCH) {
     float u[BATCH][N];
 #pragma unroll
-    for (int j = 0; j < BATCH; ++j)        // past the last segment: re-read the last one (dropped below)
-      ldcg_vec<N>(partial + (size_t)min(c + j, t.z) * cta_stride + off, u[j]);
+    for (int j = 0; j < BATCH; ++j) ldcg_vec<N>(partial + (size_t)min(c + j, t.z) * cta_stride + off, u[j]);
 #pragma unroll
     for (int j = 0; j < BATCH; ++j) {
       const bool on = c + j <= t.z;
@@ -211,14 +238,23 @@ __device__ __forceinline__ void sum_partials_cg(const float* __restrict__ partia
     }
   }
 }
+// One sum on its own.
+template <int N, int BATCH>
+__device__ __forceinline__ void sum_partials_cg(const float* __restrict__ partial, const MegaGemmShape& s, int NT, int n0,
+                                                int tok, float (&x)[N]) {
+  const int4 t = tile_seg(s, n0);
+  PartialLoads<N, BATCH> q;
+  partials_issue<N, BATCH>(partial, s, NT, t, n0, tok, q);
+  partials_sum<N, BATCH>(partial, s, NT, t, n0, tok, q, x);
+}
 
 // 1/rms of row r; warp-collective (every lane returns it).  Lane i reads slices i, i+32.
 __device__ __forceinline__ float warp_row_inv_rms(const MegaArgs& a, int r, int lane) {
-  const int ns = (a.d + kRowSlice - 1) / kRowSlice;
-  float ss = 0.f;
-  for (int i = lane; i < ns; i += 32) ss += __ldcg(a.rowss + (size_t)r * kMaxSlices + i);
-  ss = warp_sum(ss);
-  return rsqrtf(ss / a.d + a.eps);
+  const int ns = (a.d + kRowSlice - 1) / kRowSlice;        // <= 64
+  const float* p = a.rowss + (size_t)r * kMaxSlices;
+  const float v0 = lane < ns ? __ldcg(p + lane) : 0.f;
+  const float v1 = lane + 32 < ns ? __ldcg(p + lane + 32) : 0.f;
+  return rsqrtf(warp_sum(v0 + v1) / a.d + a.eps);
 }
 
 // ---- stage: embedding (or residual add) + lazy RMSNorm operand -------------------------------------
@@ -269,16 +305,17 @@ __device__ void stage_residual(const MegaArgs& a, int wtid, int mode, const Mega
 // ---- helpers shared by the stages ----------------------------------------------------------------------
 // 1/rms of every active row into shared memory: warp w takes rows w, w+8, ... (four rows' loads in flight).
 // Split in two so that a stage can put its own loads in flight between the halves.
-struct InvRmsLoads { float s[4]; };
+struct InvRmsLoads { float v[4][2]; };
 __device__ __forceinline__ InvRmsLoads inv_rms_issue(const MegaArgs& a, int r0, int lane) {
-  const int ns = (a.d + kRowSlice - 1) / kRowSlice;
+  const int ns = (a.d + kRowSlice - 1) / kRowSlice;        // <= 64: two slices per lane
   InvRmsLoads q;
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
     const int r = r0 + 8 * k;
-    q.s[k] = 0.f;
-    if (r < a.B && a.st.active[r])
-      for (int i = lane; i < ns; i += 32) q.s[k] += __ldcg(a.rowss + (size_t)r * kMaxSlices + i);
+    const bool on = r < a.B && a.st.active[r];
+    const float* p = a.rowss + (size_t)(on ? r : 0) * kMaxSlices;
+    q.v[k][0] = (on && lane < ns) ? __ldcg(p + lane) : 0.f;
+    q.v[k][1] = (on && lane + 32 < ns) ? __ldcg(p + lane + 32) : 0.f;
   }
   return q;
 }
@@ -286,7 +323,7 @@ __device__ __forceinline__ void inv_rms_finish(const MegaArgs& a, MegaSmem* sm, 
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
     const int r = r0 + 8 * k;
-    const float t = warp_sum(q.s[k]);
+    const float t = warp_sum(q.v[k][0] + q.v[k][1]);
     if (r < a.B && lane == 0) sm->inv_s[r] = a.st.active[r] ? rsqrtf(t / a.d + a.eps) : 0.f;
   }
 }
@@ -470,9 +507,17 @@ __device__ void stage_attention(const MegaArgs& a, MegaSmem* sm, int wtid, int l
         else sincosf((float)pos * a.inv_freq[(lane & 15) * EPL + j], &sn[j], &cs[j]);
       }
       float qx[EPL], kx[EPL], vx[EPL];
-      sum_partials_cg<EPL, 4>(a.partial, gs, a.NT, hd * DH + e0, r, qx);
-      sum_partials_cg<EPL, 4>(a.partial, gs, a.NT, d + hd * DH + e0, r, kx);
-      sum_partials_cg<EPL, 4>(a.partial, gs, a.NT, 2 * d + hd * DH + e0, r, vx);
+      {
+        const int nq = hd * DH + e0, nk = d + nq, nv = 2 * d + nq;
+        const int4 tq = tile_seg(gs, nq), tk = tile_seg(gs, nk), tv = tile_seg(gs, nv);
+        PartialLoads<EPL, 4> lq, lk, lv;
+        partials_issue<EPL, 4>(a.partial, gs, a.NT, tq, nq, r, lq);
+        partials_issue<EPL, 4>(a.partial, gs, a.NT, tk, nk, r, lk);
+        partials_issue<EPL, 4>(a.partial, gs, a.NT, tv, nv, r, lv);
+        partials_sum<EPL, 4>(a.partial, gs, a.NT, tq, nq, r, lq, qx);
+        partials_sum<EPL, 4>(a.partial, gs, a.NT, tk, nk, r, lk, kx);
+        partials_sum<EPL, 4>(a.partial, gs, a.NT, tv, nv, r, lv, vx);
+      }
       int pg = single ? sm->pair_pgnew[wid] : a.st.block_table[(size_t)r * a.st.max_pages + pos / kPageTokens];
       if (pg < 0 || pg >= a.kv.n_pages) { atomicCAS(a.status, 0u, (uint32_t)kStatusBadPage); pg = -1; }
       bf16* kdst = a.kv.pool + (size_t)layer * a.kv.layer_stride + (size_t)(pg < 0 ? 0 : pg) * a.kv.page_elems +
@@ -642,6 +687,16 @@ __device__ void stage_attention(const MegaArgs& a, MegaSmem* sm, int wtid, int l
 // ---- stage: SwiGLU ----------------------------------------------------------------------------------
 // 8 consecutive features per thread (two 128-bit loads per partial segment, one 128-bit store).  The loads
 // for 1/rms and the first unit's partials are in flight together.
+__device__ __forceinline__ void gate_up_sums(const MegaArgs& a, const MegaGemmShape& gs, int f0, int r, float (&gt)[8],
+                                             float (&up)[8]) {
+  const int4 tg = tile_seg(gs, f0), tu = tile_seg(gs, a.F + f0);
+  PartialLoads<8, 2> qg, qu;
+  partials_issue<8, 2>(a.partial, gs, a.NT, tg, f0, r, qg);
+  partials_issue<8, 2>(a.partial, gs, a.NT, tu, a.F + f0, r, qu);
+  partials_sum<8, 2>(a.partial, gs, a.NT, tg, f0, r, qg, gt);
+  partials_sum<8, 2>(a.partial, gs, a.NT, tu, a.F + f0, r, qu, up);
+}
+
 __device__ void stage_swiglu(const MegaArgs& a, MegaSmem* sm, int wtid) {
   const MegaGemmShape& gs = a.shape[2];
   const int lane = wtid & 31, wid = wtid >> 5;
@@ -656,10 +711,7 @@ __device__ void stage_swiglu(const MegaArgs& a, MegaSmem* sm, int wtid) {
     r = (int)(e / F8);
     f0 = (int)(e - (long long)r * F8) << 3;
     have = a.st.active[r] != 0;
-    if (have) {
-      sum_partials_cg<8, 2>(a.partial, gs, a.NT, f0, r, gt);
-      sum_partials_cg<8, 2>(a.partial, gs, a.NT, a.F + f0, r, up);
-    }
+    if (have) gate_up_sums(a, gs, f0, r, gt, up);
   }
   inv_rms_finish(a, sm, q, wid, lane);
   for (int r0 = wid + 32; r0 < a.B; r0 += 32) {
@@ -683,10 +735,7 @@ __device__ void stage_swiglu(const MegaArgs& a, MegaSmem* sm, int wtid) {
     r = (int)(e / F8);
     f0 = (int)(e - (long long)r * F8) << 3;
     have = a.st.active[r] != 0;
-    if (have) {
-      sum_partials_cg<8, 2>(a.partial, gs, a.NT, f0, r, gt);
-      sum_partials_cg<8, 2>(a.partial, gs, a.NT, a.F + f0, r, up);
-    }
+    if (have) gate_up_sums(a, gs, f0, r, gt, up);
   }
 }
 
