@@ -36,6 +36,8 @@ namespace ss {
 
 constexpr int kMegaThreads = 352;
 constexpr int kMegaWorkers = 256;          // warps 3..10
+constexpr int kMegaMaxStages = 8;          // ring depth bound (shared memory holds 5 at batch 16)
+constexpr int kSegTabEntries = 256;        // tile-table entries kept in shared memory (the four per-layer projections)
 constexpr int kRowSlice = 128;             // elements of a row handled by one residual work item (one warp, 4 per lane)
 constexpr int kMaxSlices = 64;             // d_model <= 8192
 
@@ -46,6 +48,7 @@ struct MegaGemmShape {
   int gsplit;              // CTAs that share the iteration space (the others idle through this projection)
   long long total;
   const TileSeg* tiles;
+  int smem_off;            // first entry of this projection's table in MegaSmem::seg_tab, or -1 (read it from `tiles`)
 };
 
 // Range of the (tile, k-block) iteration space owned by a CTA.
@@ -99,8 +102,8 @@ __device__ __forceinline__ unsigned long long global_timer_ns() {
 }
 
 struct MegaSmem {
-  uint64_t full[kGemmMaxStages];
-  uint64_t empty[kGemmMaxStages];
+  uint64_t full[kMegaMaxStages];
+  uint64_t empty[kMegaMaxStages];
   uint64_t acc_full[2];
   uint64_t acc_empty[2];
   uint32_t tmem_base;
@@ -117,10 +120,10 @@ struct MegaSmem {
   int pair_pos[8], pair_pgnew[8];  // new token's position and page
   int unit_pg[8][8];               // page ids of each warp's units (when it has at most 8)
   float rope_c[8][128], rope_sn[8][128];   // cos / sin of the new position per pair, cooperative lane layout
-  float red[8];
-  uint32_t am_key[2][4][64];       // per-tile arg-max scratch: [tile half][warp][batch row]
-  int am_id[2][4][64];
+  int4 seg_tab[kSegTabEntries];    // tile tables of the per-layer projections (when they fit)
+  uint8_t active_s[kMaxBatch];     // rows active in this step
 };
+static_assert(sizeof(float) * 8 * 9 * 132 >= 2 * (2 * 4 * 64 * 4), "arg-max scratch aliases att_s");
 
 __device__ __forceinline__ void named_bar_workers() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
@@ -195,8 +198,10 @@ __device__ __forceinline__ void ldcg_vec(const float* p, float (&x)[N]) {
 //   partials_issue() the first segment and the next BATCH segments (loads only, unconditional so that they
 //                    stay in registers: past the last segment the last one is read again and dropped);
 //   partials_sum()   the additions, and any segments beyond the first batch.
-__device__ __forceinline__ int4 tile_seg(const MegaGemmShape& s, int n0) {
-  return __ldg(reinterpret_cast<const int4*>(s.tiles) + n0 / kTileN);
+__device__ __forceinline__ int4 tile_seg(const MegaSmem* sm, const MegaGemmShape& s, int n0) {
+  const int tile = n0 / kTileN;
+  if (s.smem_off >= 0) return sm->seg_tab[s.smem_off + tile];
+  return __ldg(reinterpret_cast<const int4*>(s.tiles) + tile);
 }
 template <int N, int BATCH>
 struct PartialLoads {
@@ -240,9 +245,9 @@ __device__ __forceinline__ void partials_sum(const float* __restrict__ partial, 
 }
 // One sum on its own.
 template <int N, int BATCH>
-__device__ __forceinline__ void sum_partials_cg(const float* __restrict__ partial, const MegaGemmShape& s, int NT, int n0,
-                                                int tok, float (&x)[N]) {
-  const int4 t = tile_seg(s, n0);
+__device__ __forceinline__ void sum_partials_cg(const MegaSmem* sm, const float* __restrict__ partial, const MegaGemmShape& s,
+                                                int NT, int n0, int tok, float (&x)[N]) {
+  const int4 t = tile_seg(sm, s, n0);
   PartialLoads<N, BATCH> q;
   partials_issue<N, BATCH>(partial, s, NT, t, n0, tok, q);
   partials_sum<N, BATCH>(partial, s, NT, t, n0, tok, q, x);
@@ -261,14 +266,14 @@ __device__ __forceinline__ float warp_row_inv_rms(const MegaArgs& a, int r, int 
 // Work unit = (row, slice of 128 columns) per warp, 4 columns per lane; units are dealt round-robin over
 // the CTAs first, so the whole stage is one pass with a few warps busy in every CTA.
 // mode 0: h = E[cur_tok]; mode 1: h += projection (partials of shape `gs`).
-__device__ void stage_residual(const MegaArgs& a, int wtid, int mode, const MegaGemmShape* gs,
+__device__ void stage_residual(const MegaArgs& a, const MegaSmem* sm, int wtid, int mode, const MegaGemmShape* gs,
                                const bf16* __restrict__ gain, bool dump) {
   const int ns = (a.d + kRowSlice - 1) / kRowSlice;
   const int n_units = a.B * ns;
   const int lane = wtid & 31, wid = wtid >> 5;
   for (int u = wid * gridDim.x + blockIdx.x; u < n_units; u += 8 * gridDim.x) {
     const int r = u / ns, sl = u - r * ns;
-    if (!a.st.active[r]) continue;
+    if (!sm->active_s[r]) continue;
     const int c = sl * kRowSlice + lane * 4;
     float ss = 0.f;
     if (c < a.d) {
@@ -282,7 +287,7 @@ __device__ void stage_residual(const MegaArgs& a, int wtid, int mode, const Mega
         v[0] = e0.x; v[1] = e0.y; v[2] = e1.x; v[3] = e1.y;
       } else {
         const float4 h4 = __ldcg(reinterpret_cast<const float4*>(a.h + (size_t)r * a.d + c));
-        sum_partials_cg<4, 12>(a.partial, *gs, a.NT, c, r, v);
+        sum_partials_cg<4, 12>(sm, a.partial, *gs, a.NT, c, r, v);
         v[0] += h4.x; v[1] += h4.y; v[2] += h4.z; v[3] += h4.w;
       }
       const uint2 gb = __ldg(reinterpret_cast<const uint2*>(gain + c));
@@ -306,13 +311,13 @@ __device__ void stage_residual(const MegaArgs& a, int wtid, int mode, const Mega
 // 1/rms of every active row into shared memory: warp w takes rows w, w+8, ... (four rows' loads in flight).
 // Split in two so that a stage can put its own loads in flight between the halves.
 struct InvRmsLoads { float v[4][2]; };
-__device__ __forceinline__ InvRmsLoads inv_rms_issue(const MegaArgs& a, int r0, int lane) {
+__device__ __forceinline__ InvRmsLoads inv_rms_issue(const MegaArgs& a, const MegaSmem* sm, int r0, int lane) {
   const int ns = (a.d + kRowSlice - 1) / kRowSlice;        // <= 64: two slices per lane
   InvRmsLoads q;
 #pragma unroll
   for (int k = 0; k < 4; ++k) {
     const int r = r0 + 8 * k;
-    const bool on = r < a.B && a.st.active[r];
+    const bool on = r < a.B && sm->active_s[r];
     const float* p = a.rowss + (size_t)(on ? r : 0) * kMaxSlices;
     q.v[k][0] = (on && lane < ns) ? __ldcg(p + lane) : 0.f;
     q.v[k][1] = (on && lane + 32 < ns) ? __ldcg(p + lane + 32) : 0.f;
@@ -324,13 +329,13 @@ __device__ __forceinline__ void inv_rms_finish(const MegaArgs& a, MegaSmem* sm, 
   for (int k = 0; k < 4; ++k) {
     const int r = r0 + 8 * k;
     const float t = warp_sum(q.v[k][0] + q.v[k][1]);
-    if (r < a.B && lane == 0) sm->inv_s[r] = a.st.active[r] ? rsqrtf(t / a.d + a.eps) : 0.f;
+    if (r < a.B && lane == 0) sm->inv_s[r] = sm->active_s[r] ? rsqrtf(t / a.d + a.eps) : 0.f;
   }
 }
 __device__ __forceinline__ void stage_inv_rms(const MegaArgs& a, MegaSmem* sm, int wtid) {
   const int lane = wtid & 31, wid = wtid >> 5;
   for (int r0 = wid; r0 < a.B; r0 += 32) {
-    const InvRmsLoads q = inv_rms_issue(a, r0, lane);
+    const InvRmsLoads q = inv_rms_issue(a, sm, r0, lane);
     inv_rms_finish(a, sm, q, r0, lane);
   }
   named_bar_workers();
@@ -363,6 +368,14 @@ __device__ void attention_setup(const MegaArgs& a, MegaSmem* sm, int wtid) {
   constexpr int EPL = DH / 32;
   const int lane = wtid & 31, wid = wtid >> 5;
   const int H = a.H, B = a.B;
+  // ---- per-step copies in shared memory: which rows are active, and the per-layer tile tables
+  for (int r = wtid; r < kMaxBatch; r += kMegaWorkers) sm->active_s[r] = (r < B && a.st.active[r]) ? 1 : 0;
+  for (int t = 0; t < 4; ++t) {
+    const MegaGemmShape& gs = a.shape[t];
+    if (gs.smem_off < 0) continue;
+    for (int i = wtid; i < gs.n_tiles; i += kMegaWorkers)
+      sm->seg_tab[gs.smem_off + i] = __ldg(reinterpret_cast<const int4*>(gs.tiles) + i);
+  }
   // ---- pages per row (exclusive prefix, active rows only) and this CTA's run of pairs
   if (wid == 0) {
     int cnt[8], loc = 0;
@@ -509,7 +522,7 @@ __device__ void stage_attention(const MegaArgs& a, MegaSmem* sm, int wtid, int l
       float qx[EPL], kx[EPL], vx[EPL];
       {
         const int nq = hd * DH + e0, nk = d + nq, nv = 2 * d + nq;
-        const int4 tq = tile_seg(gs, nq), tk = tile_seg(gs, nk), tv = tile_seg(gs, nv);
+        const int4 tq = tile_seg(sm, gs, nq), tk = tile_seg(sm, gs, nk), tv = tile_seg(sm, gs, nv);
         PartialLoads<EPL, 4> lq, lk, lv;
         partials_issue<EPL, 4>(a.partial, gs, a.NT, tq, nq, r, lq);
         partials_issue<EPL, 4>(a.partial, gs, a.NT, tk, nk, r, lk);
@@ -687,9 +700,9 @@ __device__ void stage_attention(const MegaArgs& a, MegaSmem* sm, int wtid, int l
 // ---- stage: SwiGLU ----------------------------------------------------------------------------------
 // 8 consecutive features per thread (two 128-bit loads per partial segment, one 128-bit store).  The loads
 // for 1/rms and the first unit's partials are in flight together.
-__device__ __forceinline__ void gate_up_sums(const MegaArgs& a, const MegaGemmShape& gs, int f0, int r, float (&gt)[8],
+__device__ __forceinline__ void gate_up_sums(const MegaArgs& a, const MegaSmem* sm, const MegaGemmShape& gs, int f0, int r, float (&gt)[8],
                                              float (&up)[8]) {
-  const int4 tg = tile_seg(gs, f0), tu = tile_seg(gs, a.F + f0);
+  const int4 tg = tile_seg(sm, gs, f0), tu = tile_seg(sm, gs, a.F + f0);
   PartialLoads<8, 2> qg, qu;
   partials_issue<8, 2>(a.partial, gs, a.NT, tg, f0, r, qg);
   partials_issue<8, 2>(a.partial, gs, a.NT, tu, a.F + f0, r, qu);
@@ -703,19 +716,19 @@ __device__ void stage_swiglu(const MegaArgs& a, MegaSmem* sm, int wtid) {
   const int F8 = a.F >> 3;
   const long long n = (long long)a.B * F8, stride = (long long)gridDim.x * kMegaWorkers;
   long long e = (long long)blockIdx.x * kMegaWorkers + wtid;
-  const InvRmsLoads q = inv_rms_issue(a, wid, lane);
+  const InvRmsLoads q = inv_rms_issue(a, sm, wid, lane);
   float gt[8], up[8];
   int r = 0, f0 = 0;
   bool have = false;
   if (e < n) {
     r = (int)(e / F8);
     f0 = (int)(e - (long long)r * F8) << 3;
-    have = a.st.active[r] != 0;
-    if (have) gate_up_sums(a, gs, f0, r, gt, up);
+    have = sm->active_s[r] != 0;
+    if (have) gate_up_sums(a, sm, gs, f0, r, gt, up);
   }
   inv_rms_finish(a, sm, q, wid, lane);
   for (int r0 = wid + 32; r0 < a.B; r0 += 32) {
-    const InvRmsLoads q2 = inv_rms_issue(a, r0, lane);
+    const InvRmsLoads q2 = inv_rms_issue(a, sm, r0, lane);
     inv_rms_finish(a, sm, q2, r0, lane);
   }
   named_bar_workers();
@@ -734,8 +747,8 @@ __device__ void stage_swiglu(const MegaArgs& a, MegaSmem* sm, int wtid) {
     if (e >= n) break;
     r = (int)(e / F8);
     f0 = (int)(e - (long long)r * F8) << 3;
-    have = a.st.active[r] != 0;
-    if (have) gate_up_sums(a, gs, f0, r, gt, up);
+    have = sm->active_s[r] != 0;
+    if (have) gate_up_sums(a, sm, gs, f0, r, gt, up);
   }
 }
 
@@ -744,8 +757,9 @@ __device__ void stage_swiglu(const MegaArgs& a, MegaSmem* sm, int wtid) {
 __device__ void stage_tile_argmax(const MegaArgs& a, MegaSmem* sm, int wtid) {
   const MegaGemmShape& gs = a.shape[4];
   const int half_id = wtid >> 7, t128 = wtid & 127, lane = wtid & 31, w4 = t128 >> 5;
-  uint32_t* s_key = &sm->am_key[half_id][0][0];       // [4 warps][64 batch rows]
-  int* s_id = &sm->am_id[half_id][0][0];
+  // scratch [tile half][4 warps][64 batch rows] of keys, then of ids, in the attention partials' space
+  uint32_t* s_key = reinterpret_cast<uint32_t*>(&sm->att_s[0][0][0]) + half_id * 256;
+  int* s_id = reinterpret_cast<int*>(&sm->att_s[0][0][0]) + 512 + half_id * 256;
   stage_inv_rms(a, sm, wtid);
   const size_t slot_stride = (size_t)a.NT * kTileN, cta_stride = slot_stride * gs.max_seg;
   for (int tile0 = blockIdx.x * 2; tile0 < a.n_tiles_lm; tile0 += gridDim.x * 2) {
@@ -753,12 +767,12 @@ __device__ void stage_tile_argmax(const MegaArgs& a, MegaSmem* sm, int wtid) {
     const bool tile_ok = tile < a.n_tiles_lm;
     const int v = tile * 128 + t128;
     int4 ts = make_int4(0, 1, 0, 0);
-    if (tile_ok) ts = __ldg(reinterpret_cast<const int4*>(gs.tiles) + v / kTileN);
+    if (tile_ok) ts = tile_seg(sm, gs, v);
     for (int rb = 0; rb < a.B; rb += 64) {              // 64 batch rows at a time (scratch holds 4 x 64 per half)
       const int rend = min(a.B, rb + 64);
       for (int r = rb; r < rend; ++r) {
         uint32_t key = 0;
-        if (tile_ok && a.st.active[r] && v < a.V) {
+        if (tile_ok && sm->active_s[r] && v < a.V) {
           const size_t off = (size_t)r * kTileN + (v % kTileN);
           float lg = __ldcg(a.partial + (size_t)ts.x * slot_stride + off);
           for (int c = ts.y; c <= ts.z; ++c) lg += __ldcg(a.partial + (size_t)c * cta_stride + off);
@@ -776,7 +790,7 @@ __device__ void stage_tile_argmax(const MegaArgs& a, MegaSmem* sm, int wtid) {
       named_bar_workers();
       if (tile_ok) {
         for (int r = rb + t128; r < rend; r += 128) {
-          if (!a.st.active[r]) continue;
+          if (!sm->active_s[r]) continue;
           uint32_t bk = s_key[r - rb];
           int bi = s_id[r - rb];
 #pragma unroll
@@ -1013,7 +1027,7 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
     if (tracer) a.trace[tr++] = global_timer_ns();
     if (cta == 0 && wtid == 0) a.st.scalars[1] = 0;   // rows still active after this step (counted in the last stage)
     attention_setup<DH>(a, sm, wtid);
-    stage_residual(a, wtid, 0, nullptr, a.norm_ptr[0], a.n_layers == 0);
+    stage_residual(a, sm, wtid, 0, nullptr, a.norm_ptr[0], a.n_layers == 0);
     ok = grid_barrier(a, sm, epoch, wtid);
     if (ok && wtid == 0) sm->act_epoch = 1;
     if (tracer) a.trace[tr++] = global_timer_ns();
@@ -1071,11 +1085,11 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
       if (type == 0) {
         stage_attention<DH>(a, sm, wtid, layer);
       } else if (type == 1) {
-        stage_residual(a, wtid, 1, &a.shape[1], a.norm_ptr[2 * layer + 1], false);
+        stage_residual(a, sm, wtid, 1, &a.shape[1], a.norm_ptr[2 * layer + 1], false);
       } else if (type == 2) {
         stage_swiglu(a, sm, wtid);
       } else if (type == 3) {
-        stage_residual(a, wtid, 1, &a.shape[3], a.norm_ptr[2 * layer + 2], layer + 1 == a.n_layers);
+        stage_residual(a, sm, wtid, 1, &a.shape[3], a.norm_ptr[2 * layer + 2], layer + 1 == a.n_layers);
       } else {
         stage_tile_argmax(a, sm, wtid);
       }

@@ -440,9 +440,14 @@ int enqueue_decode_step(ss_ctx* c, const ss_step_opts* opts, int32_t* next_token
   a.inv_freq = c->inv_freq;
   const int shp[5][2] = {{3 * d, d}, {d, d}, {2 * F, d}, {d, F}, {V, d}};
   size_t need_partial = 0;
+  int tab_entries = 0;
+  for (int i = 0; i < 4; ++i) tab_entries += ceil_div(shp[i][0], kTileN);
+  int tab_off = 0;
   for (int i = 0; i < 5; ++i) {
     const DecodeSplit p = plan_decode(shp[i][0], shp[i][1], c->n_sm);
-    a.shape[i] = {p.n_tiles, p.kb, p.max_seg, p.gsplit, p.total, c->tbl[i]};
+    const int off = (i < 4 && tab_entries <= kSegTabEntries) ? tab_off : -1;   // the per-layer tables, if they fit
+    tab_off += p.n_tiles;
+    a.shape[i] = {p.n_tiles, p.kb, p.max_seg, p.gsplit, p.total, c->tbl[i], off};
     need_partial = std::max(need_partial, (size_t)p.gsplit * p.max_seg * NT * kTileN * sizeof(float));
   }
   if (need_partial > c->partial_bytes) return SS_ERR_CAPACITY;
