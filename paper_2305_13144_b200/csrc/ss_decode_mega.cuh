@@ -18,7 +18,7 @@
 //
 // Operand roles: one tcgen05.mma costs about the same issue time whatever its shape, so the decode
 // projections put the WEIGHTS on the wide side: D[token, row] += X[token, 16] . W[row, 16]^T with
-// M = 128 token lanes and N = 256 weight rows (8 KiB of weights per instruction).  Token lanes
+// M = 64 or 128 token lanes and N = 256 weight rows (8 KiB of weights per instruction).  Token lanes
 // beyond the batch compute on whatever shared memory follows the activation block; rows of D are
 // independent, and those lanes are never read.
 //
@@ -970,7 +970,8 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
   } else if (warp == 1) {
     // ===================== MMA issuer =====================
     if (lane == 0) {
-      const uint32_t idesc = umma_idesc_bf16(kTileN);     // M = 128 token lanes, N = 256 weight rows
+      // M = token lanes (64 up to 64 rows: half the tensor-core work on unused lanes), N = 256 weight rows
+      const uint32_t idesc = umma_idesc_bf16(kTileN, a.NT <= 64 ? 64 : 128);
       int gi = 0, seg = 0;
       bool ok = true;
       for (int gm = 0; gm < n_gemm && ok; ++gm) {
@@ -1053,8 +1054,10 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
         tc_fence_after();
         const size_t slot = (size_t)cta * gs.max_seg + seg_local;
         for (int mt = 0; mt < a.m_tiles; ++mt) {
-          if (mt * 128 + quarter * 32 >= a.B) continue;        // no batch row in this warp's lanes (warp-uniform)
-          const int tok = mt * 128 + quarter * 32 + lane;
+          // batch row held by this thread's lane: 32 per lane quarter, or 16 with the 64-row instruction
+          const int per_q = a.NT <= 64 ? 16 : 32;
+          if (mt * 128 + quarter * per_q >= a.B) continue;     // no batch row in this warp's lanes (warp-uniform)
+          const int tok = lane < per_q ? mt * 128 + quarter * per_q + lane : a.B;
           const uint32_t taddr =
               tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((buf + mt) * kTileN + colhalf * 128);
           float* dst = a.partial + (slot * a.NT + tok) * kTileN + colhalf * 128;

@@ -151,9 +151,11 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
   d |= (uint64_t)2 << 61;                          // layout: SWIZZLE_128B
   return d;
 }
-// Instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, M = 128, N = n.
-__host__ __device__ constexpr uint32_t umma_idesc_bf16(int n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+// Instruction descriptor: fp32 accumulate, bf16 A and B, both K-major, M = m (128 or 64), N = n.
+// Accumulator row i of an M = 128 instruction is tensor-memory lane i; of an M = 64 instruction it is lane
+// (i % 16) + 32 * (i / 16), i.e. the first 16 lanes of each warp's lane quarter.
+__host__ __device__ constexpr uint32_t umma_idesc_bf16(int n, int m = 128) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
 // ------------------------------------------------------------------------------------ split bookkeeping
