@@ -934,7 +934,7 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
         {
           const long long t0 = clock64();
           while (sm->act_epoch <= gm) {
-            __nanosleep(100);
+            __nanosleep(20);
             if (sm->abort) { ok = false; break; }
             if (clock64() - t0 > 4000000000LL) {
               atomicCAS(a.status, 0u, (uint32_t)kStatusFlagTimeout);
