@@ -358,6 +358,7 @@ __device__ __forceinline__ void group_bar(int id, int threads) {
 // load step and chunks gl, gl+GROUP, gl+2*GROUP, gl+3*GROUP, so each warp-wide load reads 64
 // contiguous bytes per key (full sectors).
 constexpr int kAttnPass = 8;               // pairs per pass (= worker warps)
+constexpr int kAttnU = 2;                  // load steps per work unit of the cache scan (one batch of loads in flight)
 constexpr int kAttnSlots = 9;              // partials per pair: one per warp + the new token
 
 // Once per step (the lengths do not change between layers): pages per row, this CTA's run of pairs, and --
@@ -366,6 +367,8 @@ constexpr int kAttnSlots = 9;              // partials per pair: one per warp + 
 template <int DH>
 __device__ void attention_setup(const MegaArgs& a, MegaSmem* sm, int wtid) {
   constexpr int EPL = DH / 32;
+  constexpr int UT = kAttnU * (32 / (DH / 32));   // cached tokens per work unit (16 at Dh 128, 32 at Dh 64)
+  constexpr int UPP = kPageTokens / UT;           // units per page
   const int lane = wtid & 31, wid = wtid >> 5;
   const int H = a.H, B = a.B;
   // ---- per-step copies in shared memory: which rows are active, and the per-layer tile tables
@@ -383,7 +386,7 @@ __device__ void attention_setup(const MegaArgs& a, MegaSmem* sm, int wtid) {
     for (int j = 0; j < 8; ++j) {
       const int r = lane * 8 + j;
       int c = 0;
-      if (r < B && a.st.active[r]) c = (a.st.ctx_len[r] + kPageTokens - 1) / kPageTokens;
+      if (r < B && a.st.active[r]) c = (a.st.ctx_len[r] + UT - 1) / UT;
       cnt[j] = c;
       loc += c;
     }
@@ -456,13 +459,20 @@ __device__ void attention_setup(const MegaArgs& a, MegaSmem* sm, int wtid) {
         sm->pair_pgnew[wid] = a.st.block_table[(size_t)r * a.st.max_pages + pos / kPageTokens];
       }
     }
+    // page ids of the first (up to 8) distinct pages of this warp's slice, in scan order
     const int u0 = (int)((long long)wid * U / 8), u1 = (int)((long long)(wid + 1) * U / 8);
-    if (lane < 8 && u0 + lane < u1) {
-      const int u = u0 + lane;
-      int j = 0;
+    const int u = u0 + lane;
+    int j = 0, ui = 0;
+    bool newpage = false;
+    if (u < u1) {
       while (j + 1 < np && sm->pair_ustart[j + 1] <= u) ++j;
-      sm->unit_pg[wid][lane] = a.st.block_table[(size_t)(sm->pair_id[j] / H) * a.st.max_pages + (u - sm->pair_ustart[j])];
+      ui = u - sm->pair_ustart[j];
+      newpage = lane == 0 || ui % UPP == 0;
     }
+    const unsigned int starts = __ballot_sync(0xffffffffu, newpage);
+    const int ord = __popc(starts & (0xffffffffu >> (31 - lane))) - 1;
+    if (newpage && ord < 8)
+      sm->unit_pg[wid][ord] = a.st.block_table[(size_t)(sm->pair_id[j] / H) * a.st.max_pages + ui / UPP];
   }
   named_bar_workers();
 }
@@ -472,8 +482,8 @@ __device__ void stage_attention(const MegaArgs& a, MegaSmem* sm, int wtid, int l
   constexpr int GROUP = DH / 32;           // lanes per key in the cache scan
   constexpr int KPW = 32 / GROUP;          // keys per warp-wide load step
   constexpr int EPL = DH / 32;             // cooperative layout: consecutive dimensions per lane
-  constexpr int STEPS = kPageTokens / KPW; // load steps per page (4 at Dh 128, 2 at Dh 64)
-  constexpr int U = 2;                     // load steps per batch
+  constexpr int U = kAttnU;                // load steps per work unit: one batch of loads
+  constexpr int UPP = kPageTokens / (U * KPW);   // units per page (2 at Dh 128, 1 at Dh 64)
   const int lane = wtid & 31, wid = wtid >> 5;
   const int gl = lane % GROUP, g = lane / GROUP;
   const int H = a.H, d = a.d, B = a.B;
@@ -594,19 +604,24 @@ __device__ void stage_attention(const MegaArgs& a, MegaSmem* sm, int wtid, int l
 #pragma unroll
         for (int e = 0; e < 32; ++e) acc[e] = 0.f;
       };
+      int kpage = -1, pg = 0;                            // ordinal of the current page in this slice, its id
       for (int u = u0; u < u1; ++u) {
         if (u >= sm->pair_ustart[j + 1]) { flush(j); ++j; }
         const int p = sm->pair_id[j];
         const int r = p / H, hd = p - r * H;
-        const int pi = u - sm->pair_ustart[j];
+        const int ui = u - sm->pair_ustart[j];           // unit of the pair: page ui / UPP, batch ui % UPP of it
+        const int pi = ui / UPP;
         const int pos = single ? sm->pair_pos[j] : a.st.ctx_len[r];
-        int pg = (single && u - u0 < 8) ? sm->unit_pg[wid][u - u0] : a.st.block_table[(size_t)r * a.st.max_pages + pi];
-        if (pg < 0 || pg >= a.kv.n_pages) { atomicCAS(a.status, 0u, (uint32_t)kStatusBadPage); pg = 0; }
+        if (u == u0 || ui % UPP == 0) {
+          ++kpage;
+          pg = (single && kpage < 8) ? sm->unit_pg[wid][kpage] : a.st.block_table[(size_t)r * a.st.max_pages + pi];
+          if (pg < 0 || pg >= a.kv.n_pages) { atomicCAS(a.status, 0u, (uint32_t)kStatusBadPage); pg = 0; }
+        }
         const int tcount = min(kPageTokens, pos - pi * kPageTokens);
         const bf16* kb = kv_layer + (size_t)pg * a.kv.page_elems + (size_t)hd * kPageTokens * DH;
         const float* qs = sm->q_s[j];
-#pragma unroll 1
-        for (int s0 = 0; s0 < STEPS; s0 += U) {
+        {
+          const int s0 = (ui % UPP) * U;
           uint4 kk[U][4], vv[U][4];
 #pragma unroll
           for (int uu = 0; uu < U; ++uu) {
