@@ -380,6 +380,20 @@ gemm_wx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
               if (c + j < n_valid) out[(size_t)(tok0 + c + j) * a.ld_out + n] = __float2bfloat16_rn(v[j]);
           }
         }
+      } else if (p.NT % 32 == 0) {
+        // read-modify-write of the fp32 residual: 32 tokens' loads in flight per round trip
+        for (int c = 0; c < p.NT; c += 32) {
+          float v[32], h[32];
+          tmem_ld32(taddr + c, v);
+          if (n < p.n_out) {
+            float* o = a.out_f32 + (size_t)(tok0 + c) * a.ld_out + n;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) h[j] = (c + j < n_valid) ? __ldcg(o + (size_t)j * a.ld_out) : 0.f;
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (c + j < n_valid) o[(size_t)j * a.ld_out] = h[j] + v[j];
+          }
+        }
       } else {
         for (int c = 0; c < p.NT; c += 8) {
           float v[8];
