@@ -7,13 +7,12 @@
 // never waits for activations, so while the other warps sit in a grid barrier or run a small
 // stage, the ring keeps filling with the next projection's weights.
 //
-// Warp roles (384 threads; warp 3 is idle, it only completes the first warp group so that the group can
-// hand its registers to the workers with setmaxnreg):
+// Warp roles (352 threads):
 //   warp 0      weight producer: linear bulk copies of 32 KiB (256-row tile, k-block) images into the ring
 //   warp 1      MMA issuer: tcgen05.mma, accumulators in tensor memory (two buffers)
 //   warp 2      activation loader: TMA loads of the [tokens x 64] activation block of each ring stage,
 //               issued once the stage that produced the activations has passed its grid barrier
-//   warps 4-11  workers: drain accumulators to fp32 partials, then run the stage between two
+//   warps 3-10  workers: drain accumulators to fp32 partials, then run the stage between two
 //               projections (partial sums in CTA order, RoPE, cache append, attention, residual,
 //               SwiGLU, arg-max, bookkeeping), separated by grid barriers
 //
@@ -35,10 +34,8 @@
 
 namespace ss {
 
-constexpr int kMegaThreads = 384;          // warp group 0: producer, MMA issuer, activation loader, one idle warp
-constexpr int kMegaWorkers = 256;          // warp groups 1 and 2 (warps 4..11)
-constexpr int kUtilRegs = 56;              // registers kept by warp group 0 ...
-constexpr int kWorkerRegs = 224;           // ... and taken by the workers (setmaxnreg; 128*40 + 256*232 <= 384*168)
+constexpr int kMegaThreads = 352;
+constexpr int kMegaWorkers = 256;          // warps 3..10
 constexpr int kMegaMaxStages = 8;          // ring depth bound (shared memory holds 5 at batch 16)
 constexpr int kSegTabEntries = 256;        // tile-table entries kept in shared memory (the four per-layer projections)
 constexpr int kRowSlice = 128;             // elements of a row handled by one residual work item (one warp, 4 per lane)
@@ -908,9 +905,6 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
   tc_fence_after();
   const uint32_t tmem_base = sm->tmem_base;
 
-  // Register hand-over: the four warps of group 0 need few registers, the cache scan of the workers many.
-  if (warp < 4) {
-  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kUtilRegs));
   if (warp == 0) {
     // ===================== weight producer =====================
     if (lane == 0) {
@@ -1033,14 +1027,12 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
         }
       }
     }
-  }
-  } else {
-    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kWorkerRegs));
+  } else if (warp >= 3) {
     // ===================== workers =====================
-    const int wtid = threadIdx.x - 128;
+    const int wtid = threadIdx.x - 96;
     const int wid = wtid >> 5;
     const int quarter = warp & 3;                   // tensor-memory lane quarter this warp may read
-    const int colhalf = wid >> 2;                   // warps 4-7 take the first 128 weight rows of a tile
+    const int colhalf = wid >> 2;                   // warps 3-6 take the first 128 weight rows of a tile
     const int acc_bufs = a.m_tiles == 1 ? 2 : 1;
     unsigned long long epoch = 0;
     int seg = 0;
