@@ -346,12 +346,13 @@ __device__ __forceinline__ void group_bar(int id, int threads) {
 }
 
 // ---- stage: q,k,v from partials + RoPE + cache append + paged attention ----------------------------------
-// Work is dealt in units of (row, head, page of 32 cached tokens).  Every CTA owns a contiguous run of
-// (row, head) pairs holding about 1/gridDim of all units (pairs are not split across CTAs, so their
-// partial results meet in shared memory).  A CTA works through its pairs in passes of up to 8:
+// Work is dealt in units of (row, head, one batch of loads = kAttnU load steps of cached tokens: 16 tokens
+// at head size 128, i.e. half a page).  Every CTA owns a contiguous run of (row, head) pairs holding
+// about 1/gridDim of all units (pairs are not split across CTAs, so their partial results meet in shared
+// memory).  A CTA works through its pairs in passes of up to 8:
 //   A  warp j builds pair j's rotated query (shared memory) and the new token's k,v: appended to the
 //      page, and entered as the pair's ninth partial (score, 1, v);
-//   B  the pass's units are cut into 8 equal contiguous slices, one per warp; a warp scans its pages
+//   B  the pass's units are cut into 8 equal contiguous slices, one per warp; a warp scans its units
 //      and leaves one (max, sum, acc) partial per pair it touched;
 //   C  warp j merges pair j's partials and writes the bf16 output.
 // Scan layout: a key row is Dh/8 chunks of 16 bytes; lane (g, gl) of the warp handles key g of the
@@ -361,9 +362,9 @@ constexpr int kAttnPass = 8;               // pairs per pass (= worker warps)
 constexpr int kAttnU = 2;                  // load steps per work unit of the cache scan (one batch of loads in flight)
 constexpr int kAttnSlots = 9;              // partials per pair: one per warp + the new token
 
-// Once per step (the lengths do not change between layers): pages per row, this CTA's run of pairs, and --
-// when the run fits one pass -- the pass list, the new tokens' positions/pages/rotations and the page ids
-// of every warp's units.
+// Once per step (the lengths do not change between layers): units per row, this CTA's run of pairs, and --
+// when the run fits one pass -- the pass list, the new tokens' positions/pages/rotations and the ids of
+// the first pages of every warp's slice.
 template <int DH>
 __device__ void attention_setup(const MegaArgs& a, MegaSmem* sm, int wtid) {
   constexpr int EPL = DH / 32;
