@@ -272,6 +272,42 @@ def run_group_13b(api, device):
             "value": arms["scheduled_fcr_vbs"]["tokens_per_s"], "arms": arms}
 
 
+def run_sweep(api, device, peak):
+    """Decode-step microbenchmark at the 7B shape over batch size and context (the paper's Fig. 3a / Fig. 6
+    axes): every row has the same prompt length, 32 decode steps are timed on the device after 8 warm-up steps;
+    bytes = weights + the cached keys/values read + the entries written."""
+    import torch
+    shape = synth.LLAMA_7B
+    kv_tok = 2 * shape.d_model * 2 * shape.n_layers
+    rt = api.runtime_cfg(256, 1024, 16384, 64, 256 * 640)
+    eng = make_engine(shape, rt, seed=1234, device=device)
+    rng = np.random.default_rng(0)
+    out = []
+    for ctx in (128, 512):
+        for B in (1, 8, 16, 32, 64, 128, 256):
+            toks = rng.integers(3, shape.vocab, size=B * ctx, dtype=np.int32)
+            cu = (np.arange(B + 1) * ctx).astype(np.int32)
+            api.ss_prefill(eng, toks, cu, np.full(B, 1 << 20, dtype=np.int32), 64)
+            api.ss_decode_steps(eng, 8)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            st = eng.stream                              # the stream the engine launches on
+            n = 32
+            e0.record(st)
+            api.ss_decode_steps(eng, n)
+            e1.record(st)
+            e1.synchronize()
+            ms = e0.elapsed_time(e1) / n
+            api.ss_release_batch(eng)
+            ctx_mid = ctx + 8 + n / 2.0                      # cached tokens per row, mid-window
+            nbytes = 13214687232 + B * ctx_mid * kv_tok + B * kv_tok
+            out.append({"B": B, "ctx": ctx, "ms_per_step": round(ms, 4), "tokens_per_s": round(B / ms * 1e3, 1),
+                        "gbs": round(nbytes / ms / 1e6, 1), "frac_of_peak": round(nbytes / ms / 1e6 / peak, 3)})
+    return {"metric": "decode step sweep", "unit": "ms/step", "n_gpus": 1, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "llama7b-shape bf16 decode steps, equal-length rows, batch x context sweep"},
+            "peak_gbs": peak, "points": out}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -283,6 +319,8 @@ def main():
     ap.add_argument("--trace", action="store_true", help="add the per-stage timing of one decode step")
     ap.add_argument("--group-13b", action="store_true",
                     help="instead of the batch-16 workload: the 13B-shape group of 512 queries, vanilla vs scheduled")
+    ap.add_argument("--sweep", action="store_true",
+                    help="instead of the batch-16 workload: decode-step time over batch size and context (7B shape)")
     ap.add_argument("--layers", type=int, default=0, help="debug: truncate the model (invalidates the number)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
@@ -308,6 +346,10 @@ def main():
     if args.group_13b:
         if rank == 0:
             print(json.dumps(run_group_13b(api, device)), flush=True)
+        return
+    if args.sweep:
+        if rank == 0:
+            print(json.dumps(run_sweep(api, device, float(measured_peaks()[0]["hbm_gbs"]))), flush=True)
         return
     shape = synth.LLAMA_7B if not args.layers else synth.LLAMA_7B.with_layers(args.layers)
     kv_tok = 2 * shape.d_model * 2 * shape.n_layers
