@@ -235,6 +235,20 @@ def test_wide_batches_span_several_token_tiles(B):
     assert el <= LOGIT_TOL and eh <= HIDDEN_TOL, (B, el, eh)
 
 
+def test_wide_ffn_reads_tile_tables_from_global_memory():
+    """A feed-forward width whose gate/up projection alone has 248 tiles of 256 rows: the four per-layer
+    tile tables (258 entries) no longer fit the decode kernel's shared-memory copy, so every stage looks its
+    partial segments up in global memory.  Head size 128, one layer, ragged batch of 5."""
+    shape = synth.ModelShape(n_layers=1, d_model=512, n_heads=4, head_dim=128, d_ffn=31744, vocab=1024)
+    w = synth.make_weights(shape, seed=33)
+    rng = np.random.default_rng(33)
+    prompts = [rng.integers(3, shape.vocab, size=int(n)).tolist() for n in (9, 33, 17, 40, 5)]
+    targets = [4, 2, 4, 3, 1]
+    el, eh = _teacher_forced(shape, w, prompts, targets, cap=4, max_batch=16, max_ctx=64, max_prefill=256,
+                             max_new=8, kv_tokens=1024)
+    assert el <= LOGIT_TOL and eh <= HIDDEN_TOL, (el, eh)
+
+
 def test_7b_shape_two_layers_sampled_rows():
     """The 7B shape (d 4096, 32 heads x 128, FFN 11008, vocab 32000) cut to two layers, batch 16 with the
     benchmark's prompt lengths; the oracle follows the three rows with the shortest prompts through the
