@@ -176,18 +176,25 @@ __device__ __forceinline__ bool grid_barrier(const MegaArgs& a, MegaSmem* sm, un
 // The stages between projections are chains of dependent L2 round trips (~0.7 us each), not bandwidth: the
 // helpers below put independent loads in flight together and keep only true dependencies serial.
 
+// An L2 load that the compiler may not move (a plain __ldcg can sink to its first use, which puts its
+// round trip back in series with the loads issued in between).
+__device__ __forceinline__ float ldcg_now(const float* p) {
+  float v;
+  asm volatile("ld.global.cg.f32 %0, [%1];" : "=f"(v) : "l"(p));
+  return v;
+}
+
 template <int N>
 __device__ __forceinline__ void ldcg_vec(const float* p, float (&x)[N]) {
   static_assert(N == 2 || N == 4 || N == 8, "N");
   if constexpr (N == 2) {
-    const float2 u = __ldcg(reinterpret_cast<const float2*>(p));
-    x[0] = u.x; x[1] = u.y;
+    asm volatile("ld.global.cg.v2.f32 {%0, %1}, [%2];" : "=f"(x[0]), "=f"(x[1]) : "l"(p));
   } else {
 #pragma unroll
-    for (int i = 0; i < N; i += 4) {
-      const float4 u = __ldcg(reinterpret_cast<const float4*>(p + i));
-      x[i] = u.x; x[i + 1] = u.y; x[i + 2] = u.z; x[i + 3] = u.w;
-    }
+    for (int i = 0; i < N; i += 4)
+      asm volatile("ld.global.cg.v4.f32 {%0, %1, %2, %3}, [%4];"
+                   : "=f"(x[i]), "=f"(x[i + 1]), "=f"(x[i + 2]), "=f"(x[i + 3])
+                   : "l"(p + i));
   }
 }
 
@@ -257,8 +264,8 @@ __device__ __forceinline__ void sum_partials_cg(const MegaSmem* sm, const float*
 __device__ __forceinline__ float warp_row_inv_rms(const MegaArgs& a, int r, int lane) {
   const int ns = (a.d + kRowSlice - 1) / kRowSlice;        // <= 64
   const float* p = a.rowss + (size_t)r * kMaxSlices;
-  const float v0 = lane < ns ? __ldcg(p + lane) : 0.f;
-  const float v1 = lane + 32 < ns ? __ldcg(p + lane + 32) : 0.f;
+  const float v0 = lane < ns ? ldcg_now(p + lane) : 0.f;
+  const float v1 = lane + 32 < ns ? ldcg_now(p + lane + 32) : 0.f;
   return rsqrtf(warp_sum(v0 + v1) / a.d + a.eps);
 }
 
@@ -319,8 +326,8 @@ __device__ __forceinline__ InvRmsLoads inv_rms_issue(const MegaArgs& a, const Me
     const int r = r0 + 8 * k;
     const bool on = r < a.B && sm->active_s[r];
     const float* p = a.rowss + (size_t)(on ? r : 0) * kMaxSlices;
-    q.v[k][0] = (on && lane < ns) ? __ldcg(p + lane) : 0.f;
-    q.v[k][1] = (on && lane + 32 < ns) ? __ldcg(p + lane + 32) : 0.f;
+    q.v[k][0] = (on && lane < ns) ? ldcg_now(p + lane) : 0.f;
+    q.v[k][1] = (on && lane + 32 < ns) ? ldcg_now(p + lane + 32) : 0.f;
   }
   return q;
 }
@@ -755,7 +762,7 @@ __device__ void stage_swiglu(const MegaArgs& a, MegaSmem* sm, int wtid) {
 #pragma unroll
       for (int j = 0; j < 8; ++j) {
         const float gv = gt[j] * inv;
-        ob[j] = __float2bfloat16_rn(gv / (1.f + __expf(-gv)) * (up[j] * inv));
+        ob[j] = __float2bfloat16_rn(__fdividef(gv, 1.f + __expf(-gv)) * (up[j] * inv));
       }
       *reinterpret_cast<uint4*>(a.act + (size_t)r * a.F + f0) = *reinterpret_cast<const uint4*>(ob);
     }
