@@ -793,21 +793,37 @@ __device__ void stage_tile_argmax(const MegaArgs& a, MegaSmem* sm, int wtid) {
     if (tile_ok) ts = tile_seg(sm, gs, v);
     for (int rb = 0; rb < a.B; rb += 64) {              // 64 batch rows at a time (scratch holds 4 x 64 per half)
       const int rend = min(a.B, rb + 64);
-      for (int r = rb; r < rend; ++r) {
-        uint32_t key = 0;
-        if (tile_ok && sm->active_s[r] && v < a.V) {
-          const size_t off = (size_t)r * kTileN + (v % kTileN);
-          float lg = __ldcg(a.partial + (size_t)ts.x * slot_stride + off);
-          for (int c = ts.y; c <= ts.z; ++c) lg += __ldcg(a.partial + (size_t)c * cta_stride + off);
-          lg *= sm->inv_s[r];
-          if (a.dump_logits) a.dump_logits[(size_t)r * a.V + v] = lg;
-          if (!(a.st.eos_at[r] > 0 && v == a.eos_id)) key = float_order_key(lg);
+      for (int r0 = rb; r0 < rend; r0 += 8) {           // 8 rows' partial loads in flight together
+        float x0[8], x1[8], x2[8];
+        const size_t col = (size_t)(v % kTileN);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int r = r0 + j;
+          const bool on = tile_ok && r < rend && sm->active_s[r] && v < a.V;
+          const size_t off = (size_t)(on ? r : 0) * kTileN + col;
+          x0[j] = on ? __ldcg(a.partial + (size_t)ts.x * slot_stride + off) : 0.f;
+          x1[j] = (on && ts.y <= ts.z) ? __ldcg(a.partial + (size_t)ts.y * cta_stride + off) : 0.f;
+          x2[j] = (on && ts.y + 1 <= ts.z) ? __ldcg(a.partial + (size_t)(ts.y + 1) * cta_stride + off) : 0.f;
         }
-        const uint32_t best = __reduce_max_sync(0xffffffffu, key);
-        const uint32_t who = __ballot_sync(0xffffffffu, key == best);
-        if (lane == 0) {
-          s_key[w4 * 64 + (r - rb)] = best;
-          s_id[w4 * 64 + (r - rb)] = tile * 128 + w4 * 32 + (__ffs(who) - 1);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int r = r0 + j;
+          if (r >= rend) break;                           // uniform over the CTA
+          uint32_t key = 0;
+          if (tile_ok && sm->active_s[r] && v < a.V) {
+            float lg = x0[j] + x1[j] + x2[j];             // CTA order: slot0, c_next, c_next + 1, ...
+            const size_t off = (size_t)r * kTileN + col;
+            for (int c = ts.y + 2; c <= ts.z; ++c) lg += __ldcg(a.partial + (size_t)c * cta_stride + off);
+            lg *= sm->inv_s[r];
+            if (a.dump_logits) a.dump_logits[(size_t)r * a.V + v] = lg;
+            if (!(a.st.eos_at[r] > 0 && v == a.eos_id)) key = float_order_key(lg);
+          }
+          const uint32_t best = __reduce_max_sync(0xffffffffu, key);
+          const uint32_t who = __ballot_sync(0xffffffffu, key == best);
+          if (lane == 0) {
+            s_key[w4 * 64 + (r - rb)] = best;
+            s_id[w4 * 64 + (r - rb)] = tile * 128 + w4 * 32 + (__ffs(who) - 1);
+          }
         }
       }
       named_bar_workers();
