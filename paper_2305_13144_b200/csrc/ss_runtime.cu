@@ -456,7 +456,7 @@ int enqueue_decode_step(ss_ctx* c, const ss_step_opts* opts, int32_t* next_token
   a.x_rows = NT > 128 ? 128 : NT;
   const int stage_bytes = kBlockBytes + a.m_tiles * a.x_rows * kTileK * 2;
   const int header = (int)sizeof(MegaSmem) + 1024;
-  a.stages = std::max(2, std::min(kGemmMaxStages, (227 * 1024 - header) / stage_bytes));
+  a.stages = std::max(2, std::min(kMegaMaxStages, (227 * 1024 - header) / stage_bytes));
   const size_t smem = (size_t)header + (size_t)a.stages * stage_bytes;
   a.st = c->st; a.kv = c->kv;
   a.h = c->h_dec; a.x = c->x_dec; a.o = c->o_dec; a.act = c->act_dec;
