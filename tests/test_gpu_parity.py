@@ -220,11 +220,11 @@ def test_errors_before_launch():
     api.ss_release_batch(eng)
 
 
-@pytest.mark.parametrize("B", [40, 64, 130])
+@pytest.mark.parametrize("B", [40, 64, 100, 130])
 def test_wide_batches_span_several_token_tiles(B):
-    """Batches wider than 16 rows: 48 and 64 rows (64-lane accumulator, all four lane quarters) and 144 (two
-    128-lane accumulator tiles), the per-tile arg-max in
-    groups of 64 rows, attention passes of more than 8 (row, head) pairs per CTA."""
+    """Batches wider than 16 rows: token tiles of 48 and 64 (64-lane accumulator, all four lane quarters),
+    112 (one 128-lane accumulator tile) and 144 (two 128-lane tiles); the per-tile arg-max in groups of 64
+    rows; attention passes of more than 8 (row, head) pairs per CTA."""
     shape = synth.TINY.with_layers(1)
     w = synth.make_weights(shape, seed=21)
     rng = np.random.default_rng(B)
