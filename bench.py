@@ -272,6 +272,27 @@ def run_group_13b(api, device):
             "value": arms["scheduled_fcr_vbs"]["tokens_per_s"], "arms": arms}
 
 
+def run_ablation(api, device):
+    """The three switches of the paper's ablation (Table 5) on the 1024-query group at the 7B shape: sorting by
+    predicted length is always on; binning (cells of 50), failure collection and recomputation (FCR), variable
+    batch size (VBS).  Vanilla random batching is the reference for the gains."""
+    shape = synth.LLAMA_7B
+    kv_tok = 2 * shape.d_model * 2 * shape.n_layers
+    eng = make_engine(shape, api.runtime_cfg(256, 768, 16384, 512, int(120e9 // kv_tok)), seed=1234, device=device)
+    g = synth.group_7b_1024(seed=0)
+    arms = {"vanilla": run_group_arm(eng, api, g, api.sched_cfg(vanilla=True), synth.make_permutation(g.n, 0))}
+    for binning, fcr, vbs in ((0, 0, 0), (0, 1, 0), (0, 1, 1), (1, 0, 0), (1, 1, 0), (1, 1, 1)):
+        cfg = api.sched_cfg(bin_size=50 if binning else 1, use_fcr=bool(fcr), use_vbs=bool(vbs),
+                            kv_budget_bytes=int(120e9) if vbs else 0, kv_bytes_per_token=kv_tok if vbs else 0)
+        name = "binning=%d fcr=%d vbs=%d" % (binning, fcr, vbs)
+        arms[name] = run_group_arm(eng, api, g, cfg, None)
+        arms[name]["gain_vs_vanilla"] = arms[name]["tokens_per_s"] / arms["vanilla"]["tokens_per_s"]
+    return {"metric": METRIC, "unit": "tokens/s", "n_gpus": 1, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "llama7b-shape bf16, 1024 queries, predicted = true + N(0,40); Table 5 switches"},
+            "value": arms["binning=1 fcr=1 vbs=1"]["tokens_per_s"], "arms": arms,
+            "paper_context": "Table 5 on one A100-80G: +42 / +44 / +82 / +30 / +52 / +86 % samples/s in the same row order"}
+
+
 def run_sweep(api, device, peak):
     """Decode-step microbenchmark at the 7B shape over batch size and context (the paper's Fig. 3a / Fig. 6
     axes): every row has the same prompt length, 32 decode steps are timed on the device after 8 warm-up steps;
@@ -319,6 +340,8 @@ def main():
     ap.add_argument("--trace", action="store_true", help="add the per-stage timing of one decode step")
     ap.add_argument("--group-13b", action="store_true",
                     help="instead of the batch-16 workload: the 13B-shape group of 512 queries, vanilla vs scheduled")
+    ap.add_argument("--ablation", action="store_true",
+                    help="instead of the batch-16 workload: binning / FCR / VBS switched one by one (1024 queries, 7B shape)")
     ap.add_argument("--sweep", action="store_true",
                     help="instead of the batch-16 workload: decode-step time over batch size and context (7B shape)")
     ap.add_argument("--layers", type=int, default=0, help="debug: truncate the model (invalidates the number)")
@@ -346,6 +369,10 @@ def main():
     if args.group_13b:
         if rank == 0:
             print(json.dumps(run_group_13b(api, device)), flush=True)
+        return
+    if args.ablation:
+        if rank == 0:
+            print(json.dumps(run_ablation(api, device)), flush=True)
         return
     if args.sweep:
         if rank == 0:
