@@ -293,6 +293,48 @@ def run_ablation(api, device):
             "paper_context": "Table 5 on one A100-80G: +42 / +44 / +82 / +30 / +52 / +86 % samples/s in the same row order"}
 
 
+def run_perception(api, device):
+    """What the length-perception pass costs against what scheduling gains (the paper's paragraph on the
+    overhead of length prediction, Sec. 4.2): every query's prompt plus a 32-token instruction suffix is
+    processed and 3 tokens are generated (the predicted number), in batches of 256, before the group is
+    scheduled; the predictions themselves are the synthetic ones (true + N(0,40))."""
+    shape = synth.LLAMA_7B
+    kv_tok = 2 * shape.d_model * 2 * shape.n_layers
+    eng = make_engine(shape, api.runtime_cfg(256, 768, 16384, 512, int(120e9 // kv_tok)), seed=1234, device=device)
+    g = synth.group_7b_1024(seed=0)
+    vanilla = run_group_arm(eng, api, g, api.sched_cfg(vanilla=True), synth.make_permutation(g.n, 0))
+    sched = run_group_arm(eng, api, g, api.sched_cfg(use_vbs=True, kv_budget_bytes=int(120e9), kv_bytes_per_token=kv_tok), None)
+    rng = np.random.Generator(np.random.Philox(7))
+    suffix = 32
+    plen = g.prompt_len + suffix
+    off = np.zeros(g.n + 1, dtype=np.int64)
+    np.cumsum(plen, out=off[1:])
+    toks = np.empty(int(off[-1]), dtype=np.int32)
+    extra = rng.integers(3, shape.vocab, size=suffix).astype(np.int32)         # the same instruction for every query
+    for i in range(g.n):
+        toks[off[i]:off[i] + g.prompt_len[i]] = g.prompt(i)
+        toks[off[i] + g.prompt_len[i]:off[i + 1]] = extra
+    three = np.full(g.n, 3, dtype=np.int32)
+    cfg = api.sched_cfg(vanilla=True, base_batch=256, max_new_tokens=4)
+    t0 = time.time()
+    res = api.ss_run_group(eng, cfg, toks, off, three, np.arange(g.n, dtype=np.int32), three)
+    wall = time.time() - t0
+    st = res["stats"]
+    perc_s = (st["prefill_ms"] + st["decode_ms"]) / 1e3
+    useful = float(g.true_len.sum())
+    return {"metric": METRIC, "unit": "tokens/s", "n_gpus": 1, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "llama7b-shape bf16, 1024 queries; perception pass = prompt + 32 tokens, 3 generated, batches of 256"},
+            "value": useful / (perc_s + sched["device_s"]),
+            "vanilla_tokens_per_s": vanilla["tokens_per_s"], "scheduled_tokens_per_s": sched["tokens_per_s"],
+            "perception": {"device_s": perc_s, "wall_s": wall, "prefill_s": st["prefill_ms"] / 1e3,
+                           "decode_s": st["decode_ms"] / 1e3, "batches": st["n_batches"], "steps": st["steps"],
+                           "prompt_tokens": int(off[-1])},
+            "scheduled_device_s": sched["device_s"], "vanilla_device_s": vanilla["device_s"],
+            "overhead_of_scheduled_run": perc_s / sched["device_s"],
+            "gain_vs_vanilla_without_perception": sched["tokens_per_s"] / vanilla["tokens_per_s"],
+            "gain_vs_vanilla_with_perception": vanilla["device_s"] / (perc_s + sched["device_s"])}
+
+
 def run_sweep(api, device, peak):
     """Decode-step microbenchmark at the 7B shape over batch size and context (the paper's Fig. 3a / Fig. 6
     axes): every row has the same prompt length, 32 decode steps are timed on the device after 8 warm-up steps;
@@ -342,6 +384,8 @@ def main():
                     help="instead of the batch-16 workload: the 13B-shape group of 512 queries, vanilla vs scheduled")
     ap.add_argument("--ablation", action="store_true",
                     help="instead of the batch-16 workload: binning / FCR / VBS switched one by one (1024 queries, 7B shape)")
+    ap.add_argument("--perception", action="store_true",
+                    help="instead of the batch-16 workload: cost of the length-perception pass against the scheduling gain")
     ap.add_argument("--sweep", action="store_true",
                     help="instead of the batch-16 workload: decode-step time over batch size and context (7B shape)")
     ap.add_argument("--layers", type=int, default=0, help="debug: truncate the model (invalidates the number)")
@@ -373,6 +417,10 @@ def main():
     if args.ablation:
         if rank == 0:
             print(json.dumps(run_ablation(api, device)), flush=True)
+        return
+    if args.perception:
+        if rank == 0:
+            print(json.dumps(run_perception(api, device)), flush=True)
         return
     if args.sweep:
         if rank == 0:
