@@ -265,40 +265,45 @@ gather_last_rmsnorm_kernel(const float* __restrict__ h, const int32_t* __restric
 }
 
 // In-place RoPE on q and k of the packed [T, 3d] projection, and copy of k,v into the pages.
-// grid (T, H), block Dh/2.  tok_row / tok_pos give each token's row in the batch and position.
-__global__ void rope_append_prefill_kernel(bf16* __restrict__ qkv, const int32_t* __restrict__ tok_row,
-                                           const int32_t* __restrict__ tok_pos, RowState st, KvLayout kv, int layer,
-                                           const float* __restrict__ inv_freq, int d, uint32_t* status) {
+// grid (T), block 256 = (256 / (Dh/2)) heads side by side x Dh/2 rotation pairs; the sine and cosine of a
+// (token, pair) are computed once and used for every head.  tok_row / tok_pos give each token's row in the
+// batch and position.
+__global__ void __launch_bounds__(256)
+rope_append_prefill_kernel(bf16* __restrict__ qkv, const int32_t* __restrict__ tok_row,
+                           const int32_t* __restrict__ tok_pos, RowState st, KvLayout kv, int layer,
+                           const float* __restrict__ inv_freq, int d, uint32_t* status) {
   pdl_launch_dependents();
   pdl_wait();
-  const int hd = blockIdx.y, i = threadIdx.x;
   const size_t t = blockIdx.x;
   const int r = tok_row[t], pos = tok_pos[t];
   const int Dh = kv.Dh, half = Dh >> 1;
-  bf16* q = qkv + t * 3 * d + hd * Dh;
-  bf16* k = q + d;
-  const bf16* v = k + d;
+  const int i = threadIdx.x % half, hsub = threadIdx.x / half, hpar = blockDim.x / half;
   float sn, cs;
   sincosf((float)pos * inv_freq[i], &sn, &cs);
-  const float q0 = __bfloat162float(q[i]), q1 = __bfloat162float(q[i + half]);
-  const float k0 = __bfloat162float(k[i]), k1 = __bfloat162float(k[i + half]);
-  const bf16 kr0 = __float2bfloat16_rn(k0 * cs - k1 * sn), kr1 = __float2bfloat16_rn(k1 * cs + k0 * sn);
-  q[i] = __float2bfloat16_rn(q0 * cs - q1 * sn);
-  q[i + half] = __float2bfloat16_rn(q1 * cs + q0 * sn);
-  k[i] = kr0;
-  k[i + half] = kr1;
   const int page = st.block_table[(size_t)r * st.max_pages + pos / kPageTokens];
   if (page < 0 || page >= kv.n_pages) {
     atomicCAS(status, 0u, (uint32_t)kStatusBadPage);
     return;
   }
-  bf16* kbase = kv.pool + (size_t)layer * kv.layer_stride + (size_t)page * kv.page_elems +
-                ((size_t)hd * kPageTokens + (pos % kPageTokens)) * Dh;
-  bf16* vbase = kbase + (size_t)kv.H * kPageTokens * Dh;
-  kbase[i] = kr0;
-  kbase[i + half] = kr1;
-  vbase[i] = v[i];
-  vbase[i + half] = v[i + half];
+  for (int hd = hsub; hd < kv.H; hd += hpar) {
+    bf16* q = qkv + t * 3 * d + hd * Dh;
+    bf16* k = q + d;
+    const bf16* v = k + d;
+    const float q0 = __bfloat162float(q[i]), q1 = __bfloat162float(q[i + half]);
+    const float k0 = __bfloat162float(k[i]), k1 = __bfloat162float(k[i + half]);
+    const bf16 kr0 = __float2bfloat16_rn(k0 * cs - k1 * sn), kr1 = __float2bfloat16_rn(k1 * cs + k0 * sn);
+    q[i] = __float2bfloat16_rn(q0 * cs - q1 * sn);
+    q[i + half] = __float2bfloat16_rn(q1 * cs + q0 * sn);
+    k[i] = kr0;
+    k[i + half] = kr1;
+    bf16* kbase = kv.pool + (size_t)layer * kv.layer_stride + (size_t)page * kv.page_elems +
+                  ((size_t)hd * kPageTokens + (pos % kPageTokens)) * Dh;
+    bf16* vbase = kbase + (size_t)kv.H * kPageTokens * Dh;
+    kbase[i] = kr0;
+    kbase[i + half] = kr1;
+    vbase[i] = v[i];
+    vbase[i + half] = v[i + half];
+  }
 }
 
 // Causal attention over one prompt, tiled: CTA = (32 queries, head, sequence); 4 threads share a
@@ -344,24 +349,44 @@ attn_prefill_kernel(const bf16* __restrict__ qkv, const int32_t* __restrict__ cu
     }
     __syncthreads();
     const int kmax = min(KT, k_end - kt0);
-    for (int j = 0; j < kmax; ++j) {
-      float dot = 0.f;
+    for (int j = 0; j < kmax; j += 4) {              // four keys per update of the running maximum
+      float dot[4];
 #pragma unroll
-      for (int e = 0; e < PART; e += 2) {
-        const float2 kk = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&s_k[j][part * PART + e]));
-        dot += q[e] * kk.x + q[e + 1] * kk.y;
+      for (int jj = 0; jj < 4; ++jj) {
+        float dsum = 0.f;
+        if (j + jj < kmax) {                         // uniform over the CTA
+#pragma unroll
+          for (int e = 0; e < PART; e += 8) {
+            float kf[8];
+            unpack8(*reinterpret_cast<const uint4*>(&s_k[j + jj][part * PART + e]), kf);
+#pragma unroll
+            for (int x = 0; x < 8; ++x) dsum += q[e + x] * kf[x];
+          }
+          dsum += __shfl_xor_sync(0xffffffffu, dsum, 1);
+          dsum += __shfl_xor_sync(0xffffffffu, dsum, 2);
+        }
+        // causal mask (uniform within the 4-thread group)
+        dot[jj] = (j + jj < kmax && kt0 + j + jj <= qpos) ? dsum : -CUDART_INF_F;
       }
-      dot += __shfl_xor_sync(0xffffffffu, dot, 1);
-      dot += __shfl_xor_sync(0xffffffffu, dot, 2);
-      if (kt0 + j <= qpos) {                        // causal mask (uniform within the 4-thread group)
-        const float mn = fmaxf(m, dot);
-        const float sc = exp2f(m - mn), pw = exp2f(dot - mn);
-        l = l * sc + pw;
+      const float mn = fmaxf(fmaxf(fmaxf(m, dot[0]), fmaxf(dot[1], dot[2])), dot[3]);
+      if (mn != -CUDART_INF_F) {
+        const float sc = exp2f(m - mn);              // 0 while nothing has been accumulated (m = -inf)
+        l *= sc;
 #pragma unroll
-        for (int e = 0; e < PART; e += 2) {
-          const float2 vv = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&s_v[j][part * PART + e]));
-          acc[e] = acc[e] * sc + pw * vv.x;
-          acc[e + 1] = acc[e + 1] * sc + pw * vv.y;
+        for (int e = 0; e < PART; ++e) acc[e] *= sc;
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) {
+          if (dot[jj] != -CUDART_INF_F) {
+            const float pw = exp2f(dot[jj] - mn);
+            l += pw;
+#pragma unroll
+            for (int e = 0; e < PART; e += 8) {
+              float vf[8];
+              unpack8(*reinterpret_cast<const uint4*>(&s_v[j + jj][part * PART + e]), vf);
+#pragma unroll
+              for (int x = 0; x < 8; ++x) acc[e + x] += pw * vf[x];
+            }
+          }
         }
         m = mn;
       }
@@ -375,16 +400,22 @@ attn_prefill_kernel(const bf16* __restrict__ qkv, const int32_t* __restrict__ cu
   }
 }
 
-// act[t][f] = silu(gu[t][f]) * gu[t][F+f] over T tokens.  grid (T, ceil(F/256))
+// act[t][f] = silu(gu[t][f]) * gu[t][F+f] over T tokens, 8 features per thread (F a multiple of 8).
+// grid (T, ceil(F / 2048)), block 256.
 __global__ void __launch_bounds__(256)
 swiglu_kernel(const bf16* __restrict__ gu, bf16* __restrict__ act, int F) {
   pdl_launch_dependents();
   pdl_wait();
   const size_t t = blockIdx.x;
-  const int f = blockIdx.y * blockDim.x + threadIdx.x;
-  if (f >= F) return;
-  const float gt = __bfloat162float(gu[t * 2 * F + f]), up = __bfloat162float(gu[t * 2 * F + F + f]);
-  act[t * F + f] = __float2bfloat16_rn(gt / (1.f + __expf(-gt)) * up);
+  const int f0 = (blockIdx.y * blockDim.x + threadIdx.x) * 8;
+  if (f0 >= F) return;
+  float gt[8], up[8];
+  unpack8(*reinterpret_cast<const uint4*>(gu + t * 2 * F + f0), gt);
+  unpack8(*reinterpret_cast<const uint4*>(gu + t * 2 * F + F + f0), up);
+  __align__(16) bf16 ob[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) ob[j] = __float2bfloat16_rn(gt[j] / (1.f + __expf(-gt[j])) * up[j]);
+  *reinterpret_cast<uint4*>(act + t * F + f0) = *reinterpret_cast<const uint4*>(ob);
 }
 
 }  // namespace ss

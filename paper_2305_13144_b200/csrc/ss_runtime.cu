@@ -500,7 +500,7 @@ int enqueue_prefill_chunk(ss_ctx* c, int s0, int s1, const int32_t* cu, int T) {
   for (int l = 0; l < m.n_layers; ++l) {
     const LayerWeights& w = c->layers[l];
     if ((rc = run_gemm(c, w.wqkv, *mx, p_qkv, kGemmDirectBf16, T, c->qkv, nullptr, 3 * d))) return rc;
-    SS_CUDA(c, launch(c, rope_append_prefill_kernel, dim3(T, H), dim3(Dh / 2), 0, c->qkv, (const int32_t*)c->d_tok_row,
+    SS_CUDA(c, launch(c, rope_append_prefill_kernel, dim3(T), dim3(256), 0, c->qkv, (const int32_t*)c->d_tok_row,
                       (const int32_t*)c->d_tok_pos, c->st, c->kv, l, (const float*)c->inv_freq, d, c->status));
     const dim3 ag(ceil_div(max_len, 32), H, nseq);
     if (Dh == 128)
@@ -510,7 +510,7 @@ int enqueue_prefill_chunk(ss_ctx* c, int s0, int s1, const int32_t* cu, int T) {
     if ((rc = run_gemm(c, w.wo, *mo, p_o, kGemmDirectF32Add, T, nullptr, c->h, d))) return rc;
     SS_CUDA(c, launch(c, rmsnorm_kernel, dim3(T), dim3(256), 0, (const float*)c->h, (const bf16*)w.ffn_norm, c->x, d, m.rms_eps));
     if ((rc = run_gemm(c, w.wgu, *mx, p_gu, kGemmDirectBf16, T, c->gu, nullptr, 2 * F))) return rc;
-    SS_CUDA(c, launch(c, swiglu_kernel, dim3(T, ceil_div(F, 256)), dim3(256), 0, (const bf16*)c->gu, c->act, F));
+    SS_CUDA(c, launch(c, swiglu_kernel, dim3(T, ceil_div(F, 2048)), dim3(256), 0, (const bf16*)c->gu, c->act, F));
     if ((rc = run_gemm(c, w.wdown, *ma, p_dn, kGemmDirectF32Add, T, nullptr, c->h, d))) return rc;
     if (l + 1 < m.n_layers)
       SS_CUDA(c, launch(c, rmsnorm_kernel, dim3(T), dim3(256), 0, (const float*)c->h,
