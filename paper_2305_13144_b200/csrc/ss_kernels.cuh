@@ -306,32 +306,62 @@ rope_append_prefill_kernel(bf16* __restrict__ qkv, const int32_t* __restrict__ t
   }
 }
 
-// Causal attention over one prompt, tiled: CTA = (32 queries, head, sequence); 4 threads share a
-// query (a quarter of the head each); keys/values are staged through shared memory 32 at a time.
-// qkv: [T, 3d] with RoPE applied; out: [T, d].
+// Causal attention over one prompt on the tensor cores (warp-level mma, m16n8k16, bf16 in, fp32 out).
+// CTA = (64 queries, head, sequence), four warps of 16 queries; keys and values are staged through shared
+// memory 32 at a time (values transposed, so that both B operands are read as pairs of consecutive
+// elements); online softmax on the accumulator fragments; the probabilities are re-used in registers as the
+// A operand of P.V.  qkv: [T, 3d] with RoPE applied; out: [T, d].
+// Fragment layout of mma.m16n8k16 (g = lane / 4, q = lane % 4): A regs 0..3 hold rows g, g+8, g, g+8 and
+// columns 2q..2q+1 (regs 0,1) or 2q+8..2q+9 (regs 2,3); B regs 0,1 hold k = 2q..2q+1 and 2q+8..2q+9 of
+// column g; C regs 0,1 hold row g, columns 2q..2q+1, regs 2,3 row g+8.
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+               "{%0, %1, %2, %3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+
 template <int DH>
 __global__ void __launch_bounds__(128)
 attn_prefill_kernel(const bf16* __restrict__ qkv, const int32_t* __restrict__ cu_seqlens, bf16* __restrict__ out, int d) {
-  constexpr int QT = 32, KT = 32, PART = DH / 4;
-  __shared__ __align__(16) bf16 s_k[KT][DH];
-  __shared__ __align__(16) bf16 s_v[KT][DH];
+  constexpr int QT = 64, KT = 32, KS = DH / 16, NB = DH / 8;
+  constexpr int KPAD = DH + 8;                     // padded rows: conflict-free fragment loads
+  constexpr int VPAD = KT + 8;
+  __shared__ __align__(16) bf16 s_k[KT][KPAD];     // [key][dim]
+  __shared__ __align__(16) bf16 s_vt[DH][VPAD];    // [dim][key]
   pdl_launch_dependents();
   pdl_wait();
   const int hd = blockIdx.y, s = blockIdx.z;
   const int seq0 = cu_seqlens[s], len = cu_seqlens[s + 1] - seq0;
   const int qt0 = blockIdx.x * QT;
   if (qt0 >= len) return;
-  const int qi = threadIdx.x >> 2, part = threadIdx.x & 3;
-  const int qpos = qt0 + qi;
-  const bool qvalid = qpos < len;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = lane >> 2, q4 = lane & 3;
+  const int row0 = qt0 + warp * 16 + g, row1 = row0 + 8;     // this thread's two query positions
   const float qscale = rsqrtf((float)DH) * 1.4426950408889634f;
-  float q[PART], acc[PART];
+
+  // Q fragments, kept for the whole kernel (rows beyond the prompt read row len-1: valid memory, never stored)
+  uint32_t qa[KS][4];
+  {
+    const bf16* q0 = qkv + (size_t)(seq0 + min(row0, len - 1)) * 3 * d + hd * DH + q4 * 2;
+    const bf16* q1 = qkv + (size_t)(seq0 + min(row1, len - 1)) * 3 * d + hd * DH + q4 * 2;
 #pragma unroll
-  for (int j = 0; j < PART; ++j) {
-    q[j] = qvalid ? __bfloat162float(qkv[(size_t)(seq0 + qpos) * 3 * d + hd * DH + part * PART + j]) * qscale : 0.f;
-    acc[j] = 0.f;
+    for (int ks = 0; ks < KS; ++ks) {
+      qa[ks][0] = *reinterpret_cast<const uint32_t*>(q0 + ks * 16);
+      qa[ks][1] = *reinterpret_cast<const uint32_t*>(q1 + ks * 16);
+      qa[ks][2] = *reinterpret_cast<const uint32_t*>(q0 + ks * 16 + 8);
+      qa[ks][3] = *reinterpret_cast<const uint32_t*>(q1 + ks * 16 + 8);
+    }
   }
-  float m = -CUDART_INF_F, l = 0.f;
+  float o[NB][4];
+#pragma unroll
+  for (int nb = 0; nb < NB; ++nb) { o[nb][0] = o[nb][1] = o[nb][2] = o[nb][3] = 0.f; }
+  float m0 = -CUDART_INF_F, m1 = -CUDART_INF_F, l0 = 0.f, l1 = 0.f;
+
   const int k_end = min(len, qt0 + QT);            // causal: keys up to the tile's last query
   for (int kt0 = 0; kt0 < k_end; kt0 += KT) {
     __syncthreads();
@@ -345,58 +375,93 @@ attn_prefill_kernel(const bf16* __restrict__ qkv, const int32_t* __restrict__ cu
         uv = *reinterpret_cast<const uint4*>(base + d);
       }
       *reinterpret_cast<uint4*>(&s_k[kr][cc * 8]) = uk;
-      *reinterpret_cast<uint4*>(&s_v[kr][cc * 8]) = uv;
+      const bf16* pv = reinterpret_cast<const bf16*>(&uv);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) s_vt[cc * 8 + e][kr] = pv[e];
     }
     __syncthreads();
-    const int kmax = min(KT, k_end - kt0);
-    for (int j = 0; j < kmax; j += 4) {              // four keys per update of the running maximum
-      float dot[4];
+    if (kt0 > qt0 + warp * 16 + 15) continue;      // every key of the tile is after this warp's last query
+
+    // S = Q K^T for 16 queries x 32 keys
+    float sc[KT / 8][4];
 #pragma unroll
-      for (int jj = 0; jj < 4; ++jj) {
-        float dsum = 0.f;
-        if (j + jj < kmax) {                         // uniform over the CTA
+    for (int nb = 0; nb < KT / 8; ++nb) {
+      sc[nb][0] = sc[nb][1] = sc[nb][2] = sc[nb][3] = 0.f;
 #pragma unroll
-          for (int e = 0; e < PART; e += 8) {
-            float kf[8];
-            unpack8(*reinterpret_cast<const uint4*>(&s_k[j + jj][part * PART + e]), kf);
-#pragma unroll
-            for (int x = 0; x < 8; ++x) dsum += q[e + x] * kf[x];
-          }
-          dsum += __shfl_xor_sync(0xffffffffu, dsum, 1);
-          dsum += __shfl_xor_sync(0xffffffffu, dsum, 2);
-        }
-        // causal mask (uniform within the 4-thread group)
-        dot[jj] = (j + jj < kmax && kt0 + j + jj <= qpos) ? dsum : -CUDART_INF_F;
+      for (int ks = 0; ks < KS; ++ks) {
+        const uint32_t b0 = *reinterpret_cast<const uint32_t*>(&s_k[nb * 8 + g][ks * 16 + q4 * 2]);
+        const uint32_t b1 = *reinterpret_cast<const uint32_t*>(&s_k[nb * 8 + g][ks * 16 + q4 * 2 + 8]);
+        mma_bf16_16816(sc[nb], qa[ks], b0, b1);
       }
-      const float mn = fmaxf(fmaxf(fmaxf(m, dot[0]), fmaxf(dot[1], dot[2])), dot[3]);
-      if (mn != -CUDART_INF_F) {
-        const float sc = exp2f(m - mn);              // 0 while nothing has been accumulated (m = -inf)
-        l *= sc;
+    }
+    // scale, causal / length mask, running maxima
+    float mx0 = m0, mx1 = m1;
 #pragma unroll
-        for (int e = 0; e < PART; ++e) acc[e] *= sc;
+    for (int nb = 0; nb < KT / 8; ++nb) {
 #pragma unroll
-        for (int jj = 0; jj < 4; ++jj) {
-          if (dot[jj] != -CUDART_INF_F) {
-            const float pw = exp2f(dot[jj] - mn);
-            l += pw;
+      for (int e = 0; e < 2; ++e) {
+        const int key = kt0 + nb * 8 + q4 * 2 + e;
+        sc[nb][e] = (key <= row0 && key < len) ? sc[nb][e] * qscale : -CUDART_INF_F;
+        sc[nb][2 + e] = (key <= row1 && key < len) ? sc[nb][2 + e] * qscale : -CUDART_INF_F;
+        mx0 = fmaxf(mx0, sc[nb][e]);
+        mx1 = fmaxf(mx1, sc[nb][2 + e]);
+      }
+    }
+    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+    mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+    mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+    const float r0s = (mx0 == -CUDART_INF_F) ? 1.f : exp2f(m0 - mx0);     // exp2f(-inf) = 0 on the first tile
+    const float r1s = (mx1 == -CUDART_INF_F) ? 1.f : exp2f(m1 - mx1);
+    m0 = mx0;
+    m1 = mx1;
+    l0 *= r0s;
+    l1 *= r1s;
 #pragma unroll
-            for (int e = 0; e < PART; e += 8) {
-              float vf[8];
-              unpack8(*reinterpret_cast<const uint4*>(&s_v[j + jj][part * PART + e]), vf);
+    for (int nb = 0; nb < NB; ++nb) {
+      o[nb][0] *= r0s; o[nb][1] *= r0s;
+      o[nb][2] *= r1s; o[nb][3] *= r1s;
+    }
+    // probabilities, as A fragments of P V (two 16-key steps)
+    uint32_t pa[KT / 16][4];
 #pragma unroll
-              for (int x = 0; x < 8; ++x) acc[e + x] += pw * vf[x];
-            }
-          }
-        }
-        m = mn;
+    for (int nb = 0; nb < KT / 8; ++nb) {
+      float p[4];
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        p[e] = (sc[nb][e] == -CUDART_INF_F) ? 0.f : exp2f(sc[nb][e] - m0);
+        p[2 + e] = (sc[nb][2 + e] == -CUDART_INF_F) ? 0.f : exp2f(sc[nb][2 + e] - m1);
+      }
+      l0 += p[0] + p[1];
+      l1 += p[2] + p[3];
+      pa[nb >> 1][(nb & 1) * 2 + 0] = pack_bf16x2(p[0], p[1]);
+      pa[nb >> 1][(nb & 1) * 2 + 1] = pack_bf16x2(p[2], p[3]);
+    }
+    // O += P V
+#pragma unroll
+    for (int nb = 0; nb < NB; ++nb) {
+#pragma unroll
+      for (int kk = 0; kk < KT / 16; ++kk) {
+        const uint32_t b0 = *reinterpret_cast<const uint32_t*>(&s_vt[nb * 8 + g][kk * 16 + q4 * 2]);
+        const uint32_t b1 = *reinterpret_cast<const uint32_t*>(&s_vt[nb * 8 + g][kk * 16 + q4 * 2 + 8]);
+        mma_bf16_16816(o[nb], pa[kk], b0, b1);
       }
     }
   }
-  if (qvalid) {
-    const float inv = 1.f / l;
+  // row sums over the four lanes of a row, then the output
+  l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
+  l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+  l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
+  l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+  const float i0 = 1.f / l0, i1 = 1.f / l1;
 #pragma unroll
-    for (int j = 0; j < PART; ++j)
-      out[(size_t)(seq0 + qpos) * d + hd * DH + part * PART + j] = __float2bfloat16_rn(acc[j] * inv);
+  for (int nb = 0; nb < NB; ++nb) {
+    if (row0 < len)
+      *reinterpret_cast<uint32_t*>(out + (size_t)(seq0 + row0) * d + hd * DH + nb * 8 + q4 * 2) =
+          pack_bf16x2(o[nb][0] * i0, o[nb][1] * i0);
+    if (row1 < len)
+      *reinterpret_cast<uint32_t*>(out + (size_t)(seq0 + row1) * d + hd * DH + nb * 8 + q4 * 2) =
+          pack_bf16x2(o[nb][2] * i1, o[nb][3] * i1);
   }
 }
 

@@ -502,7 +502,7 @@ int enqueue_prefill_chunk(ss_ctx* c, int s0, int s1, const int32_t* cu, int T) {
     if ((rc = run_gemm(c, w.wqkv, *mx, p_qkv, kGemmDirectBf16, T, c->qkv, nullptr, 3 * d))) return rc;
     SS_CUDA(c, launch(c, rope_append_prefill_kernel, dim3(T), dim3(256), 0, c->qkv, (const int32_t*)c->d_tok_row,
                       (const int32_t*)c->d_tok_pos, c->st, c->kv, l, (const float*)c->inv_freq, d, c->status));
-    const dim3 ag(ceil_div(max_len, 32), H, nseq);
+    const dim3 ag(ceil_div(max_len, 64), H, nseq);
     if (Dh == 128)
       SS_CUDA(c, launch(c, attn_prefill_kernel<128>, ag, dim3(128), 0, (const bf16*)c->qkv, (const int32_t*)c->d_cu, c->attn_o, d));
     else
