@@ -127,6 +127,7 @@ static_assert(sizeof(float) * 8 * 9 * 132 >= 2 * (2 * 4 * 64 * 4), "arg-max scra
 
 __device__ __forceinline__ void named_bar_workers() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
+__device__ __forceinline__ void fence_proxy_async_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
 __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
   unsigned long long v;
   asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
@@ -149,9 +150,13 @@ __device__ __forceinline__ bool mega_wait(uint32_t bar, uint32_t parity, MegaSme
   }
 }
 
-// Workers only.  Returns false if the CTA aborted.
-__device__ __forceinline__ bool grid_barrier(const MegaArgs& a, MegaSmem* sm, unsigned long long& epoch, int wtid) {
-  fence_proxy_async_all();                 // activations written here are read by TMA elsewhere
+// Workers only.  Returns false if the CTA aborted.  `wrote_operand`: this CTA wrote activations that other
+// CTAs read with TMA after the barrier, so its global writes are ordered before the async proxy's reads.
+// The barrier after a projection publishes only fp32 partials, which are read with ordinary loads: there the
+// proxy fence is left out (with bulk copies of the weight ring in flight it took about 2 us per barrier).
+__device__ __forceinline__ bool grid_barrier(const MegaArgs& a, MegaSmem* sm, unsigned long long& epoch, int wtid,
+                                             bool wrote_operand) {
+  if (wrote_operand) fence_proxy_async_global();
   named_bar_workers();
   ++epoch;
   if (wtid == 0) {
@@ -1068,7 +1073,7 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
     if (cta == 0 && wtid == 0) a.st.scalars[1] = 0;   // rows still active after this step (counted in the last stage)
     attention_setup<DH>(a, sm, wtid);
     stage_residual(a, sm, wtid, 0, nullptr, a.norm_ptr[0], a.n_layers == 0);
-    ok = grid_barrier(a, sm, epoch, wtid);
+    ok = grid_barrier(a, sm, epoch, wtid, true);
     if (ok && wtid == 0) sm->act_epoch = 1;
     if (tracer) a.trace[tr++] = global_timer_ns();
 
@@ -1120,7 +1125,7 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
       }
       if (!ok) break;
       if (tracer) a.trace[tr++] = global_timer_ns();       // this CTA's accumulators drained
-      ok = grid_barrier(a, sm, epoch, wtid);
+      ok = grid_barrier(a, sm, epoch, wtid, false);
       if (!ok) break;
       if (tracer) a.trace[tr++] = global_timer_ns();       // every CTA's partials visible
       // ---- the stage that consumes the projection
@@ -1136,7 +1141,7 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
         stage_tile_argmax(a, sm, wtid);
       }
       if (tracer) a.trace[tr++] = global_timer_ns();       // this CTA's share of the stage done
-      ok = grid_barrier(a, sm, epoch, wtid);
+      ok = grid_barrier(a, sm, epoch, wtid, true);
       if (!ok) break;
       if (tracer) a.trace[tr++] = global_timer_ns();       // stage complete everywhere
       if (type == 4) stage_final(a, wtid);
