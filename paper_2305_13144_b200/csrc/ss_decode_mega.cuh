@@ -1105,14 +1105,15 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
           const uint32_t taddr =
               tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((buf + mt) * kTileN + colhalf * 128);
           float* dst = a.partial + (slot * a.NT + tok) * kTileN + colhalf * 128;
+          // 64 columns per TMEM load: the last segment's drain is the serial tail of every projection
 #pragma unroll 1
-          for (int c = 0; c < 128; c += 32) {
-            float v[32];
-            tmem_ld32(taddr + c, v);
+          for (int c = 0; c < 128; c += 64) {
+            uint32_t v[64];
+            tmem_ld64(taddr + c, v);
             if (tok < a.B) {
 #pragma unroll
-              for (int j = 0; j < 32; j += 4)
-                *reinterpret_cast<float4*>(dst + c + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+              for (int j = 0; j < 64; j += 4)
+                *reinterpret_cast<uint4*>(dst + c + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
             }
           }
         }
