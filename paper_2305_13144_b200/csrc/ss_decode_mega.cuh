@@ -126,7 +126,6 @@ struct MegaSmem {
 static_assert(sizeof(float) * 8 * 9 * 132 >= 2 * (2 * 4 * 64 * 4), "arg-max scratch aliases att_s");
 
 __device__ __forceinline__ void named_bar_workers() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
-__device__ __forceinline__ void fence_proxy_async_all() { asm volatile("fence.proxy.async;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
 __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long long* p) {
   unsigned long long v;
@@ -989,7 +988,7 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
           }
           if (!ok) break;
           __threadfence();
-          fence_proxy_async_all();
+          fence_proxy_async_global();          // global only: the full fence stalls ~2 us while ring copies are in flight
         }
         for (long long it = it0; it < it1; ++it, ++gi) {
           const long long t0 = clock64();
