@@ -987,7 +987,9 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
             }
           }
           if (!ok) break;
-          __threadfence();
+          // the worker that set the flag had acquired the grid barrier at gpu scope and released the flag at CTA
+          // scope; a CTA-scope fence here completes the chain (a gpu-scope fence costs a round trip to L2)
+          __threadfence_block();
           fence_proxy_async_global();          // global only: the full fence stalls ~2 us while ring copies are in flight
         }
         for (long long it = it0; it < it1; ++it, ++gi) {
@@ -1073,7 +1075,7 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
     attention_setup<DH>(a, sm, wtid);
     stage_residual(a, sm, wtid, 0, nullptr, a.norm_ptr[0], a.n_layers == 0);
     ok = grid_barrier(a, sm, epoch, wtid, true);
-    if (ok && wtid == 0) sm->act_epoch = 1;
+    if (ok && wtid == 0) { __threadfence_block(); sm->act_epoch = 1; }
     if (tracer) a.trace[tr++] = global_timer_ns();
 
     for (int gm = 0; gm < n_gemm && ok; ++gm) {
@@ -1145,7 +1147,7 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
       if (!ok) break;
       if (tracer) a.trace[tr++] = global_timer_ns();       // stage complete everywhere
       if (type == 4) stage_final(a, wtid);
-      else if (wtid == 0) sm->act_epoch = gm + 2;
+      else if (wtid == 0) { __threadfence_block(); sm->act_epoch = gm + 2; }
     }
   }
 
