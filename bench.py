@@ -42,7 +42,7 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one decode-step launch, from the ncu captures summarised in
 # profiles/decode_step_mega_7b_shape_ncu_full.md (2- and 4-layer cases, scaled to 32 layers).  Set to None
 # whenever the kernel changes after the capture.
-TRAFFIC_BYTES_PER_DECODE_STEP = 14.77e9
+TRAFFIC_BYTES_PER_DECODE_STEP = 14.73e9
 
 
 def measured_peaks():
