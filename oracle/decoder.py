@@ -38,6 +38,8 @@ from __future__ import annotations
 import math
 import numpy as np
 
+from .sampler import sample_token
+
 
 # ----------------------------------------------------------------------------- operators
 
@@ -220,9 +222,12 @@ class KVDecoder:
 # ----------------------------------------------------------------------------- generation
 
 def generate(model: Decoder, prompt, cap: int, eos_at: int | None = None,
-             keep_logits: bool = False, keep_hidden: bool = False) -> dict:
-    """Greedy generation of one row, at most `cap` new tokens (the first one, produced by
-    the prompt's forward pass, counts).
+             keep_logits: bool = False, keep_hidden: bool = False,
+             temperature: float = 0.0, seed: int = 0, row_key: int = 0) -> dict:
+    """Generation of one row, at most `cap` new tokens (the first one, produced by the prompt's
+    forward pass, counts).  Greedy by default; with temperature > 0 the t-th token is the draw
+    (seed, row_key, t) from softmax(logits / temperature) as defined in oracle/sampler.py
+    (Sec. 4.2: the paper generates at temperature 0.5).
 
     Termination rules (they make lengths controllable with random weights):
       * eos_at is None: natural EOS -- the row ends when argmax picks eos_id.
@@ -241,7 +246,10 @@ def generate(model: Decoder, prompt, cap: int, eos_at: int | None = None,
             logs.append(logits)
         if keep_hidden:
             hids.append(hidden)
-        tok = select_token(logits, model.eos_id, suppress_eos=eos_at is not None)
+        if temperature > 0:
+            tok = sample_token(logits, temperature, seed, row_key, t, model.eos_id, suppress_eos=eos_at is not None)
+        else:
+            tok = select_token(logits, model.eos_id, suppress_eos=eos_at is not None)
         if eos_at is not None and t == eos_at:
             tok = model.eos_id
         out.append(tok)
