@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the sequence-scheduling decode engine.
 
-    python bench.py --gpus N --steps K --warmup W [--impl reference] [--group-arms]
+    python bench.py --gpus N --steps K --warmup W [--impl reference] [--no-group]
 
 One "step" = one pass of the whole hot path over one micro-batch: ss_run_group() on the
 LLaMA-7B-shaped decoder (random bf16 weights) with a single vanilla micro-batch of 16 queries
@@ -12,11 +12,13 @@ around the prompt pass and the decode loop, inputs resident); `e2e` is the same 
 wall clock of the C-ABI call with host buffers in and out.  `roofline` is the decode loop's
 algorithmic HBM bytes (weights once per step + cached keys/values of the active rows + the
 entries written) over its device time, against the measured copy bandwidth.
-With --group-arms the 1024-query group is also run once per arm (vanilla batching, sequence
-scheduling with FCR, and FCR + variable batch size) and reported under "group".
+After the timed steps (N = 1) the 1024-query group is run once per arm -- vanilla random batching,
+sequence scheduling with FCR, and FCR + variable batch size -- and reported under "group" with the
+gain over vanilla; each arm's batch log is checked against the scheduler oracle (--no-group skips this).
 
 N > 1: the path does not shard (one GPU per engine), so ranks run independent replicas on
-different seeds; value = tokens of all ranks / slowest rank's time.
+different seeds; value = tokens of all ranks / slowest rank's time.  Without a launcher in the
+environment, --gpus N starts the N worker processes itself.
 """
 from __future__ import annotations
 
@@ -39,10 +41,32 @@ from paper_2305_13144_b200 import synth  # noqa: E402
 METRIC = "generated tokens/s"
 WORKLOAD = "llama7b-shape bf16, one vanilla micro-batch of 16, prompts U[64,256], responses lognormal(120,0.7)<=512"
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one decode-step launch, from the ncu captures summarised in
-# profiles/decode_step_mega_7b_shape_ncu_full.md (2- and 4-layer cases, scaled to 32 layers).  Set to None
-# whenever the kernel changes after the capture.
-TRAFFIC_BYTES_PER_DECODE_STEP = 14.73e9
+NOMINAL_HBM_GBS = 8000.0
+KERNEL_SOURCES = ("ss_decode_mega.cuh", "ss_gemm.cuh", "ss_kernels.cuh", "ss_internal.h")
+
+
+def kernel_sources_sha16() -> str:
+    """Fingerprint of the decode kernel's sources, to tell whether stored profiler counters still describe it."""
+    import hashlib
+    h = hashlib.sha256()
+    for name in KERNEL_SOURCES:
+        with open(os.path.join(ROOT, "paper_2305_13144_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def measured_traffic_bytes():
+    """DRAM bytes (read + write) of one decode-step launch as counted by the profiler, or None when no
+    capture of the kernel as it stands now has been recorded (the record carries the sources' fingerprint)."""
+    p = os.path.join(ROOT, "profiles", "decode_step_mega_7b_shape_traffic.json")
+    try:
+        with open(p) as f:
+            rec = json.load(f)
+        if rec.get("kernel_sources_sha16") == kernel_sources_sha16():
+            return float(rec["dram_bytes_per_launch"])
+    except Exception:
+        pass
+    return None
 
 
 def measured_peaks():
@@ -140,27 +164,37 @@ def make_engine(shape, rt, seed, device):
 
 def _oracle_sample():
     """The oracle as it stands (numpy, fp32 here) on a bounded sample of the benchmark workload: all 16 rows of
-    the batch, 16 generated tokens each (prompt pass included), 2 of the 32 layers; returns a closure that runs
-    the sample once and the factor that scales its time to the full depth."""
+    the batch, 16 generated tokens each (prompt pass included), on the 7B shape cut to 1 layer and to 2 layers.
+    Returns a closure that runs both once and gives (tokens, seconds scaled to the full depth): the difference
+    of the two runs is one layer's time, the rest (embedding, final norm, LM head, token choice) counts once."""
     from oracle import decoder as od
-    L_s, cap = 2, 16
-    shape = synth.LLAMA_7B.with_layers(L_s)
-    w = synth.make_weights(shape, seed=1234)
-    model = od.Decoder(w, n_layers=L_s, n_heads=shape.n_heads, head_dim=shape.head_dim, rms_eps=shape.rms_eps,
-                       rope_theta=shape.rope_theta, eos_id=shape.eos_id, dtype=np.float32)
-    del w
+    cap = 16
     g = synth.group_7b_batch16(seed=0)
     prompts = [g.prompt(i).tolist() for i in range(g.n)]
+    w2 = synth.make_weights(synth.LLAMA_7B.with_layers(2), seed=1234)
+    models = []
+    for L_s in (1, 2):
+        shape = synth.LLAMA_7B.with_layers(L_s)
+        models.append(od.Decoder(w2, n_layers=L_s, n_heads=shape.n_heads, head_dim=shape.head_dim,
+                                 rms_eps=shape.rms_eps, rope_theta=shape.rope_theta, eos_id=shape.eos_id,
+                                 dtype=np.float32))
+    del w2
+    L = synth.LLAMA_7B.n_layers
 
     def run():
-        t = time.time()
-        res = od.run_micro_batch(model, prompts, cap, [cap] * g.n)
-        return sum(len(r["tokens"]) for r in res["rows"]), time.time() - t
+        secs, tokens = [], 0
+        for m in models:
+            t = time.time()
+            res = od.run_micro_batch(m, prompts, cap, [cap] * g.n)
+            secs.append(time.time() - t)
+            tokens = sum(len(r["tokens"]) for r in res["rows"])
+        per_layer = max(secs[1] - secs[0], 0.0)
+        const = max(secs[0] - per_layer, 0.0)
+        return tokens, const + L * per_layer, sum(secs)
 
-    scale = synth.LLAMA_7B.n_layers / L_s
-    what = (f"all {g.n} rows, {cap} generated tokens each (prompt pass included), {L_s} of 32 layers timed in fp32 "
-            f"and scaled x{scale:g} (embedding and LM head are scaled with them, a small over-count)")
-    return run, scale, what
+    what = (f"all {g.n} rows, {cap} generated tokens each (prompt pass included), timed in fp32 on the 7B shape cut "
+            f"to 1 and to 2 layers: one layer's time = the difference, x{L} layers, plus the rest once")
+    return run, what
 
 
 def run_reference(args, rank):
@@ -168,15 +202,15 @@ def run_reference(args, rank):
     if rank != 0:
         return
     t0 = time.time()
-    run, scale, what = _oracle_sample()
+    run, what = _oracle_sample()
     setup_s = time.time() - t0
     cores = os.cpu_count()
     times, tokens = [], 0
     for it in range(args.warmup + args.steps):
-        tokens, dt = run()
+        tokens, full_s, _ = run()
         if it >= args.warmup:
-            times.append(dt)
-    sec = statistics.mean(times) * scale
+            times.append(full_s)
+    sec = statistics.mean(times)
     value = tokens / sec
     sample = f"{what}; numpy on {cores} threads; setup {setup_s:.0f}s untimed"
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
@@ -189,11 +223,11 @@ def run_reference(args, rank):
 
 
 def cpu_baseline_leg():
-    run, scale, what = _oracle_sample()
-    tokens, dt = run()
+    run, what = _oracle_sample()
+    tokens, full_s, spent = run()
     cores = os.cpu_count()
-    return {"value": tokens / (dt * scale), "unit": "tokens/s", "cores": cores, "kind": "oracle",
-            "sample": f"{what}; {dt:.1f}s of CPU time; numpy on {cores} threads"}
+    return {"value": tokens / full_s, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+            "sample": f"{what}; {spent:.1f}s of CPU time; numpy on {cores} threads"}
 
 
 def aggregate(tokens_local: float, seconds_local: float, dist):
@@ -215,11 +249,13 @@ def stage_trace(eng, api, g, steps=60):
     import torch
     cu = np.zeros(g.n + 1, dtype=np.int32)
     cu[1:] = np.cumsum(g.prompt_len)
+    api.ss_set_trace(eng, True)
     api.ss_prefill(eng, g.prompt_tokens, cu, g.true_len, 512)
     api.ss_decode_steps(eng, steps)
     torch.cuda.synchronize()
     tr = api.ss_step_trace(eng).astype(np.int64)
     api.ss_release_batch(eng)
+    api.ss_set_trace(eng, False)
     tr = tr - tr[0]
     ev = tr[2:].reshape(-1, 4)
     names = ["qkv", "o", "gate_up", "down"]
@@ -237,10 +273,33 @@ def stage_trace(eng, api, g, steps=60):
     return out
 
 
-def run_group_arm(eng, api, g, cfg, perm):
+def check_against_scheduler_oracle(res, g, cfg, perm):
+    """Checker (outside every timed region): the batch log the engine reports must equal the scheduler oracle's
+    simulation of the same group -- order, failure list, and rows / cap / steps / failures of every batch."""
+    from oracle import scheduler as osch
+    ocfg = osch.SchedCfg(bin_size=cfg.bin_size, base_batch=cfg.base_batch, use_vbs=bool(cfg.use_vbs),
+                         use_fcr=bool(cfg.use_fcr), vbs_len_threshold=cfg.vbs_len_threshold,
+                         vbs_token_budget=cfg.vbs_token_budget, min_batch=cfg.min_batch, max_batch=cfg.max_batch,
+                         max_new_tokens=cfg.max_new_tokens, kv_budget_bytes=cfg.kv_budget_bytes,
+                         kv_bytes_per_token=cfg.kv_bytes_per_token, vanilla=bool(cfg.vanilla))
+    sim = osch.simulate(g.prompt_len, g.pred_len, g.true_len, ocfg, perm)
+    order, n, nf = res["order"], g.n, len(sim["failures"])
+    assert order[:n].tolist() == sim["order"] and order[n:n + nf].tolist() == sim["failures"]
+    assert len(res["log"]) == len(sim["batches"])
+    for rec, ob in zip(res["log"], sim["batches"]):
+        assert order[rec["first_row"]:rec["first_row"] + rec["n_rows"]].tolist() == ob.rows
+        assert (rec["cap"], rec["steps"], rec["n_failed"], rec["is_recompute"]) == \
+               (ob.cap, ob.steps, len(ob.failed), int(ob.is_recompute))
+    assert res["len"].tolist() == g.true_len.tolist()
+    return sim
+
+
+def run_group_arm(eng, api, g, cfg, perm, check=True):
     t0 = time.time()
     res = api.ss_run_group(eng, cfg, g.prompt_tokens, g.prompt_off, g.pred_len, perm, g.true_len)
     wall = time.time() - t0
+    if check:
+        check_against_scheduler_oracle(res, g, cfg, perm)
     st = res["stats"]
     dev_s = (st["prefill_ms"] + st["decode_ms"]) / 1e3
     return {"tokens_per_s": st["useful_tokens"] / dev_s, "samples_per_s": g.n / dev_s,
@@ -248,8 +307,44 @@ def run_group_arm(eng, api, g, cfg, perm):
             "prefill_s": st["prefill_ms"] / 1e3, "decode_s": st["decode_ms"] / 1e3,
             "batches": st["n_batches"], "steps": st["steps"], "avg_len": st["steps"] / max(1, st["n_batches"]),
             "redundancy": 1.0 - st["useful_tokens"] / max(1, st["row_steps"]),
-            "failure_ratio": st["n_failed"] / g.n,
+            "failure_ratio": st["n_failed"] / g.n, "log_equals_scheduler_oracle": bool(check),
             "decode_gbs": st["model_bytes"] / (st["decode_ms"] / 1e3) / 1e9 if st["decode_ms"] > 0 else None}
+
+
+def run_group_arms_7b(eng, api, kv_tok):
+    """Configurations 3 and 4: the 1024-query group at the 7B shape, once per arm -- vanilla random batching,
+    sequence scheduling with bins of 50 + FCR at batch 16, and the same with variable batch size (16..256 rows
+    inside a 120 GB key/value budget)."""
+    g3 = synth.group_7b_1024(seed=0)
+    arms = {}
+    arms["vanilla"] = run_group_arm(eng, api, g3, api.sched_cfg(vanilla=True), synth.make_permutation(g3.n, 0))
+    arms["scheduled_fcr"] = run_group_arm(eng, api, g3, api.sched_cfg(), None)
+    arms["scheduled_fcr_vbs"] = run_group_arm(
+        eng, api, g3, api.sched_cfg(use_vbs=True, kv_budget_bytes=int(120e9), kv_bytes_per_token=kv_tok), None)
+    for k in ("scheduled_fcr", "scheduled_fcr_vbs"):
+        arms[k]["gain_vs_vanilla"] = arms[k]["tokens_per_s"] / arms["vanilla"]["tokens_per_s"]
+    return {"workload": "llama7b-shape bf16, 1024 queries, prompts U[64,256], responses lognormal(120,0.7)<=512, "
+                        "predicted = true + N(0,40), bins of 50", "arms": arms,
+            "paper_context": "+86% samples/s on one A100-80G (Table 4), not comparable hardware"}
+
+
+def spawn_replicas(n: int) -> int:
+    """`--gpus N` without a launcher: start one worker process per GPU (this script again, with the rank in the
+    environment), pass rank 0's JSON line through, return the first non-zero exit code."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    procs = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__)] + sys.argv[1:], env=env))
+    rc = 0
+    for p in procs:
+        p.wait()
+        rc = rc or p.returncode
+    return rc
 
 
 def run_group_13b(api, device):
@@ -377,7 +472,9 @@ def main():
     ap.add_argument("--steps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--group-arms", action="store_true", help="also run the 1024-query group: vanilla vs scheduled")
+    ap.add_argument("--no-group", action="store_true",
+                    help="skip the 1024-query group arms (vanilla vs scheduled) that follow the timed batch-16 steps")
+    ap.add_argument("--group-arms", action="store_true", help="kept for old command lines: the arms now run by default")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--trace", action="store_true", help="add the per-stage timing of one decode step")
     ap.add_argument("--group-13b", action="store_true",
@@ -399,6 +496,8 @@ def main():
     if args.impl == "reference":
         run_reference(args, rank)
         return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_replicas(args.gpus))
 
     import torch
     import torch.distributed as dist
@@ -428,7 +527,8 @@ def main():
         return
     shape = synth.LLAMA_7B if not args.layers else synth.LLAMA_7B.with_layers(args.layers)
     kv_tok = 2 * shape.d_model * 2 * shape.n_layers
-    if args.group_arms:
+    with_group = not args.no_group and not args.layers and world == 1
+    if with_group:
         kv_pool = int(120e9 // kv_tok)
         rt = api.runtime_cfg(256, 768, 16384, 512, kv_pool)
     else:
@@ -476,6 +576,7 @@ def main():
         achieved = model_bytes / decode_s / 1e9
         h2d = int(g.prompt_tokens.nbytes + 4 * (g.n + 1) + 4 * g.n + 8 * 4 * 256 + 4 * 16 * 24 + 3 * g.prompt_tokens.nbytes)
         d2h = int(tokens * 4 + 2 * 4 * g.n + 4)
+        traffic = measured_traffic_bytes() if shape.n_layers == 32 else None
         line = {
             "metric": METRIC, "value": tok_all / dev_all, "unit": "tokens/s", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": dev_all / args.steps * 1e3,
@@ -486,7 +587,8 @@ def main():
             "gpu_launches": int(launches),
             "roofline": {"bound": "hbm", "kernel": "decode_step_mega_kernel (one persistent cooperative launch per decode step)",
                          "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "peak_source": which, "traffic": TRAFFIC_BYTES_PER_DECODE_STEP if shape.n_layers == 32 else None,
+                         "peak_source": which, "peak_nominal": NOMINAL_HBM_GBS, "frac_nominal": achieved / NOMINAL_HBM_GBS,
+                         "target_frac": 0.70, "meets_target": bool(achieved / peak >= 0.70), "traffic": traffic,
                          "ms_per_decode_step": decode_s / max(1, steps_dec) * 1e3,
                          "bytes_per_decode_step": model_bytes / max(1, steps_dec)},
             "phases": {"prefill_s_per_step": prefill_s / args.steps, "decode_s_per_step": decode_s / args.steps,
@@ -495,17 +597,8 @@ def main():
         }
         if args.trace:
             line["stage_trace"] = stage_trace(eng, api, g)
-        if args.group_arms:
-            g3 = synth.group_7b_1024(seed=0)
-            arms = {}
-            arms["vanilla"] = run_group_arm(eng, api, g3, api.sched_cfg(vanilla=True), synth.make_permutation(g3.n, 0))
-            arms["scheduled_fcr"] = run_group_arm(eng, api, g3, api.sched_cfg(), None)
-            arms["scheduled_fcr_vbs"] = run_group_arm(
-                eng, api, g3, api.sched_cfg(use_vbs=True, kv_budget_bytes=int(120e9), kv_bytes_per_token=kv_tok), None)
-            for k in ("scheduled_fcr", "scheduled_fcr_vbs"):
-                arms[k]["gain_vs_vanilla"] = arms[k]["tokens_per_s"] / arms["vanilla"]["tokens_per_s"]
-            line["group"] = {"workload": "1024 queries, predicted = true + N(0,40), bins of 50", "arms": arms,
-                             "paper_context": "+86% samples/s on one A100-80G (Table 4), not comparable hardware"}
+        if with_group:
+            line["group"] = run_group_arms_7b(eng, api, kv_tok)
         if not args.no_cpu_baseline and world == 1:
             line["cpu_baseline"] = cpu_baseline_leg()
         print(json.dumps(line), flush=True)

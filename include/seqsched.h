@@ -99,6 +99,8 @@ typedef struct {
                                    token instead of its own choice (finished rows ignore it) */
   float* dump_logits;           /* device fp32 [B, vocab]: the logits the choice was made on  */
   float* dump_hidden;           /* device fp32 [B, d_model]: residual stream before the last norm */
+  int32_t* dump_choice;         /* device int32 [B]: the row's own choice (arg-max or draw), before a forced
+                                   EOS or a forced token replaces it; written for active rows only */
 } ss_step_opts;
 
 /* Per-batch record written by ss_run_group(). */
@@ -166,6 +168,21 @@ int ss_schedule(const ss_sched_cfg* cfg, const int32_t* prompt_len, const int32_
 int ss_prefill(ss_ctx* ctx, const int32_t* tokens, const int32_t* cu_seqlens, int32_t B,
                const int32_t* eos_at, int32_t cap, const ss_step_opts* opts, int32_t* first_tokens);
 
+/* Sampled decoding (Sec. 4.2, "Experimental Setting": the paper generates at temperature 0.5; Sec. 3.2: the
+ * spread of response lengths between generations).  temperature = 0 (the default) is greedy.  With
+ * temperature T > 0 the t-th generated token of a row is a draw from softmax(logits / T), taken as
+ *     argmax_v ( logit_v / T - log(-log(u_v)) ),   u_v = ((w >> 9) + 0.5) / 2^23,
+ * where w is the first output word of Philox4x32-10 (Salmon et al., SC'11) at counter (v, t, row key, 0) and key
+ * (seed & 0xffffffff, seed >> 32); ties go to the lowest id and a suppressed EOS is left out.  The draw depends
+ * only on (seed, row key, t, logits): a row regenerated from its prompt repeats its tokens.  Applies to
+ * every batch started afterwards.  SS_ERR_ARG for a negative or non-finite temperature. */
+int ss_set_sampling(ss_ctx* ctx, float temperature, uint64_t seed);
+
+/* Row keys of the NEXT ss_prefill() only (host int32 [n], n = that batch's row count): the third counter word
+ * of the draws above.  Without this call the rows of a batch have keys 0, 1, 2, ...; ss_run_group() uses each
+ * row's query index.  Infrastructure of the sampling above, no passage of its own. */
+int ss_set_row_keys(ss_ctx* ctx, const int32_t* keys, int32_t n);
+
 /* One decode step for every active row (App. D: one token per step against the cached keys
  * and values): feed the row's last token at its next position, append its key/value, attend
  * over the row's own cache (per-row length; finished rows are skipped), project, pick the
@@ -228,17 +245,35 @@ int ss_step_model_bytes(const ss_ctx* ctx, const int32_t* ctx_len, const uint8_t
  * shared-memory limit; make that first call, with the device current, before any stream capture.
  * All calls share the one array and it keeps what the last call left there (the call clears the
  * only word that must start at zero), so two calls whose kernels may overlap on the GPU --
- * different streams, or threads -- race; keep calls on one device in one stream order. */
+ * different streams, or threads -- race; keep calls on one device in one stream order.
+ * The call is asynchronous: it returns once its three kernels are enqueued.  SS_ERR_CUDA means a
+ * launch was refused (an error that the caller's earlier work left pending is discarded on entry
+ * and not reported here).  Should a bounded wait inside the projection kernel give up, every
+ * element of `logits` is set to NaN instead of a sum of incomplete partials. */
 int ss_logits_noalloc(const float* hidden, const void* norm_gain, const void* lm_head, int32_t n_rows,
                       int32_t d_model, int32_t vocab, float rms_eps, float* logits, void* stream);
 
-/* Tracing (App. D measures per-token time; this shows where one decode step spends it).  Copies the
- * time stamps (nanoseconds of the GPU's global timer) that CTA 0 took during the LAST decode step:
+/* Failure detection.  Every wait inside a kernel (on a barrier between the SMs, on a copy, on the tensor
+ * cores) is bounded: when the limit runs out the kernel records which wait it was, all of its roles leave, and the
+ * next ss_read_batch() / ss_run_group() returns SS_ERR_DEVICE_TIMEOUT (once; the context is then usable again).
+ * ss_set_wait_limit_ms() sets that limit (default about 2000 ms; 1..60000).
+ * ss_selftest_wait_timeout() demonstrates the path without putting any work at risk: it launches one small
+ * kernel in which every SM waits, for at most limit_us microseconds, for an arrival that never comes, and returns
+ * what the runtime then reports -- SS_ERR_DEVICE_TIMEOUT when detection works.  SS_ERR_STATE while a batch is in
+ * flight.  Infrastructure, no passage of the paper. */
+int ss_set_wait_limit_ms(ss_ctx* ctx, int32_t ms);
+int ss_selftest_wait_timeout(ss_ctx* ctx, int32_t limit_us);
+
+/* Tracing (App. D measures per-token time; this shows where one decode step spends it).  Off by default;
+ * ss_set_trace(ctx, 1) makes every following decode step record its stage boundaries. */
+int ss_set_trace(ss_ctx* ctx, int32_t on);
+
+/* Copies the time stamps (nanoseconds of the GPU's global timer) that CTA 0 took during the LAST decode step:
  * out[0] start, out[1] first operand ready, then for each projection in execution order
  * (qkv, o, gate/up, down per layer, LM head) four stamps: own accumulators drained, all partials
  * visible, own share of the following stage done, stage complete on every SM.
  * out: host uint64 [cap]; n receives the number of stamps (2 + 4 * (4 * n_layers + 1));
- * SS_ERR_CAPACITY if cap is smaller.  Synchronises the stream. */
+ * SS_ERR_CAPACITY if cap is smaller, SS_ERR_STATE if tracing is off.  Synchronises the stream. */
 int ss_step_trace(ss_ctx* ctx, uint64_t* out, int32_t cap, int32_t* n);
 
 const char* ss_strerror(int code);

@@ -12,11 +12,11 @@ leg may use this file; it imports nothing from the CUDA package.
 
 Readings taken where the paper is silent or garbled (each is also listed in the design
 notes of the repository):
-  * the VBS formula is printed as B0*L/L0, but the text around it ("larger batch size for
-    shorter responses", "same number of tokens in each batch") and the constants of the
-    experiments (256*50/L) fix B = B0*L0/L;
+  * the VBS formula is printed as B0*L/L0, but the paragraph around it (Sec. 4.1, Variable Batch
+    Size: shorter responses get bigger batches so that every batch holds about as many tokens)
+    and the constants of the experiments (256*50/L, Sec. 4.2) fix B = B0*L0/L;
   * an exact multiple of the cell stays in its cell (100 -> 100); predictions < 1 clamp to 1;
-  * "nearest power of 2" is by linear distance, a tie goes down;
+  * the power of two nearest to 256*50/L (Sec. 4.2) is taken by linear distance, a tie goes down;
   * the threshold rule wins over the formula at L >= 300 (batch 16 although 12800/300 = 42.7);
   * a batch may straddle bins; the allowance of its longest (latest) row governs its size;
   * the sort is ascending and stable in the original index;
@@ -63,7 +63,8 @@ class Batch:
 
 
 def bin_of(x: int, cfg: SchedCfg) -> int:
-    """Round a length up to its cell ("the nearest bin that is greater")."""
+    """Round a length up to its cell (Sec. 4.1, Binning: a length goes to the closest cell boundary at
+    or above it)."""
     x = min(max(int(x), 1), cfg.max_new_tokens)
     if cfg.bin_size == 1:
         return x

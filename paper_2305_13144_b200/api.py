@@ -23,7 +23,7 @@ EXPORTS = [
     "ss_arena_bytes", "ss_create", "ss_destroy", "ss_load_weights", "ss_schedule", "ss_prefill",
     "ss_decode_step", "ss_decode_steps", "ss_read_batch", "ss_release_batch", "ss_run_group",
     "ss_step_model_bytes", "ss_strerror", "ss_last_device_status", "ss_last_cuda_error", "ss_kernel_launches",
-    "ss_logits_noalloc", "ss_step_trace",
+    "ss_logits_noalloc", "ss_step_trace", "ss_set_trace", "ss_set_sampling", "ss_set_row_keys", "ss_set_wait_limit_ms", "ss_selftest_wait_timeout",
 ]
 
 
@@ -59,7 +59,8 @@ class ss_tensor_desc(C.Structure):
 
 
 class ss_step_opts(C.Structure):
-    _fields_ = [("forced_tokens", C.c_void_p), ("dump_logits", C.c_void_p), ("dump_hidden", C.c_void_p)]
+    _fields_ = [("forced_tokens", C.c_void_p), ("dump_logits", C.c_void_p), ("dump_hidden", C.c_void_p),
+                ("dump_choice", C.c_void_p)]
 
 
 class ss_batch_log(C.Structure):
@@ -105,6 +106,11 @@ def lib() -> C.CDLL:
         L.ss_step_model_bytes.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(C.c_double)]
         L.ss_last_device_status.argtypes = [C.c_void_p, C.POINTER(C.c_uint32)]
         L.ss_step_trace.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(C.c_int32)]
+        L.ss_set_trace.argtypes = [C.c_void_p, C.c_int32]
+        L.ss_set_wait_limit_ms.argtypes = [C.c_void_p, C.c_int32]
+        L.ss_selftest_wait_timeout.argtypes = [C.c_void_p, C.c_int32]
+        L.ss_set_sampling.argtypes = [C.c_void_p, C.c_float, C.c_uint64]
+        L.ss_set_row_keys.argtypes = [C.c_void_p, C.c_void_p, C.c_int32]
         L.ss_logits_noalloc.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32,
                                         C.c_float, C.c_void_p, C.c_void_p]
         _lib_handle = L
@@ -229,24 +235,24 @@ def ss_schedule(cfg: ss_sched_cfg, prompt_len, pred_len, perm=None):
     return order[:n], [(b.first_row, b.n_rows, b.cap, b.is_recompute) for b in batches[:nb.value]]
 
 
-def _opts(forced_tokens=None, dump_logits=None, dump_hidden=None):
-    if forced_tokens is None and dump_logits is None and dump_hidden is None:
+def _opts(forced_tokens=None, dump_logits=None, dump_hidden=None, dump_choice=None):
+    if forced_tokens is None and dump_logits is None and dump_hidden is None and dump_choice is None:
         return None
-    return ss_step_opts(_dp(forced_tokens), _dp(dump_logits), _dp(dump_hidden))
+    return ss_step_opts(_dp(forced_tokens), _dp(dump_logits), _dp(dump_hidden), _dp(dump_choice))
 
 
 def ss_prefill(ctx: Ctx, tokens, cu_seqlens, eos_at, cap: int, *, forced_tokens=None, dump_logits=None,
-               dump_hidden=None, first_tokens=None) -> None:
+               dump_hidden=None, dump_choice=None, first_tokens=None) -> None:
     tk, cu, ea = _np(tokens, np.int32), _np(cu_seqlens, np.int32), _np(eos_at, np.int32)
-    o = _opts(forced_tokens, dump_logits, dump_hidden)
+    o = _opts(forced_tokens, dump_logits, dump_hidden, dump_choice)
     _check(lib().ss_prefill(ctx.handle, _hp(tk), _hp(cu), int(cu.shape[0]) - 1, _hp(ea), int(cap),
                             C.byref(o) if o else None, _dp(first_tokens)), "ss_prefill", ctx)
 
 
-def ss_decode_step(ctx: Ctx, *, forced_tokens=None, dump_logits=None, dump_hidden=None, next_tokens=None,
-                   n_active_host=None) -> None:
+def ss_decode_step(ctx: Ctx, *, forced_tokens=None, dump_logits=None, dump_hidden=None, dump_choice=None,
+                   next_tokens=None, n_active_host=None) -> None:
     """n_active_host: pinned int32 torch tensor (host) or None."""
-    o = _opts(forced_tokens, dump_logits, dump_hidden)
+    o = _opts(forced_tokens, dump_logits, dump_hidden, dump_choice)
     nah = None if n_active_host is None else C.c_void_p(n_active_host.data_ptr())
     _check(lib().ss_decode_step(ctx.handle, C.byref(o) if o else None, _dp(next_tokens), nah), "ss_decode_step", ctx)
 
@@ -306,6 +312,28 @@ def ss_last_device_status(ctx: Ctx) -> int:
     out = C.c_uint32(0)
     _check(lib().ss_last_device_status(ctx.handle, C.byref(out)), "ss_last_device_status", ctx)
     return out.value
+
+
+def ss_set_sampling(ctx: Ctx, temperature: float, seed: int = 0) -> None:
+    _check(lib().ss_set_sampling(ctx.handle, float(temperature), int(seed)), "ss_set_sampling", ctx)
+
+
+def ss_set_row_keys(ctx: Ctx, keys) -> None:
+    k = _np(keys, np.int32)
+    _check(lib().ss_set_row_keys(ctx.handle, _hp(k), int(k.shape[0])), "ss_set_row_keys", ctx)
+
+
+def ss_set_wait_limit_ms(ctx: Ctx, ms: int) -> None:
+    _check(lib().ss_set_wait_limit_ms(ctx.handle, int(ms)), "ss_set_wait_limit_ms", ctx)
+
+
+def ss_selftest_wait_timeout(ctx: Ctx, limit_us: int) -> int:
+    """Returns the code the runtime reports after a wait that cannot complete (SS_ERR_DEVICE_TIMEOUT)."""
+    return int(lib().ss_selftest_wait_timeout(ctx.handle, int(limit_us)))
+
+
+def ss_set_trace(ctx: Ctx, on: bool) -> None:
+    _check(lib().ss_set_trace(ctx.handle, int(bool(on))), "ss_set_trace", ctx)
 
 
 def ss_step_trace(ctx: Ctx) -> np.ndarray:

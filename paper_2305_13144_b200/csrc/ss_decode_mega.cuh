@@ -88,11 +88,14 @@ struct MegaArgs {
   const int32_t* forced;
   int32_t* next_tokens;
   float *dump_logits, *dump_hidden;
+  int32_t* dump_choice;
+  SampleCfg sample;
   // sync
   unsigned long long* grid_ctr;    // monotone arrival counter
   unsigned long long grid_base;    // its value when this launch starts
   uint32_t* status;
   unsigned long long* trace;       // [2 + 4 * projections] global-timer stamps of CTA 0 (stage boundaries)
+  long long wait_limit;            // SM cycles after which any wait inside the kernel gives up
 };
 
 __device__ __forceinline__ unsigned long long global_timer_ns() {
@@ -134,19 +137,35 @@ __device__ __forceinline__ unsigned long long ld_acquire_u64(const unsigned long
 }
 
 // mbarrier wait that also gives up when the CTA aborts.
-__device__ __forceinline__ bool mega_wait(uint32_t bar, uint32_t parity, MegaSmem* sm, uint32_t* status, uint32_t code) {
+__device__ __forceinline__ bool mega_wait(uint32_t bar, uint32_t parity, MegaSmem* sm, uint32_t* status, uint32_t code,
+                                          long long limit) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
     if (mbar_try_wait(bar, parity)) return true;
     if (sm->abort) return false;
-    if (clock64() - t0 > 4000000000LL) {
+    if (clock64() - t0 > limit) {
       atomicCAS(status, 0u, code);
       sm->abort = 1;
       return false;
     }
     __nanosleep(40);                 // a spinning role must not starve the warps that share its scheduler
   }
+}
+
+// Arrival on a grid-wide counter and the bounded poll for `target` arrivals, as one thread of a CTA does them.
+// Returns false when the limit ran out (or the CTA's abort flag went up) before the counter got there.
+__device__ __forceinline__ bool arrive_and_poll(unsigned long long* ctr, unsigned long long target, long long limit,
+                                                const volatile int* abort_flag) {
+  // arrive: release-add without waiting for the old value (the writes of the whole CTA, made visible to this
+  // thread by the bar.sync in front, are ordered before it); then poll with acquire loads
+  asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(ctr), "l"(1ULL) : "memory");
+  const long long t0 = clock64();
+  while (ld_acquire_u64(ctr) < target) {
+    if (abort_flag && *abort_flag) return false;
+    if (clock64() - t0 > limit) return false;
+  }
+  return true;
 }
 
 // Workers only.  Returns false if the CTA aborted.  `wrote_operand`: this CTA wrote activations that other
@@ -159,18 +178,10 @@ __device__ __forceinline__ bool grid_barrier(const MegaArgs& a, MegaSmem* sm, un
   named_bar_workers();
   ++epoch;
   if (wtid == 0) {
-    // arrive: release-add without waiting for the old value (the writes of the whole CTA, seen through the
-    // bar.sync above, are ordered before it); then poll with acquire loads
-    asm volatile("red.release.gpu.global.add.u64 [%0], %1;" ::"l"(a.grid_ctr), "l"(1ULL) : "memory");
     const unsigned long long target = a.grid_base + epoch * gridDim.x;
-    const long long t0 = clock64();
-    while (ld_acquire_u64(a.grid_ctr) < target) {
-      if (sm->abort) break;
-      if (clock64() - t0 > 4000000000LL) {
-        atomicCAS(a.status, 0u, (uint32_t)kStatusGridBarrierTimeout);
-        sm->abort = 1;
-        break;
-      }
+    if (!arrive_and_poll(a.grid_ctr, target, a.wait_limit, &sm->abort) && !sm->abort) {
+      atomicCAS(a.status, 0u, (uint32_t)kStatusGridBarrierTimeout);
+      sm->abort = 1;
     }
   }
   named_bar_workers();
@@ -566,7 +577,7 @@ __device__ void stage_attention(const MegaArgs& a, MegaSmem* sm, int wtid, int l
         const float pq = __shfl_xor_sync(0xffffffffu, xq, 16), pk = __shfl_xor_sync(0xffffffffu, xk, 16);
         const float oq = (lane < 16) ? xq * cs[j] - pq * sn[j] : xq * cs[j] + pq * sn[j];
         const float ok = (lane < 16) ? xk * cs[j] - pk * sn[j] : xk * cs[j] + pk * sn[j];
-        const float qf = __bfloat162float(__float2bfloat16_rn(oq)) * qscale;
+        const float qf = oq * qscale;                     // the query is only ever an ALU operand: it stays fp32
         const bf16 kb16 = __float2bfloat16_rn(ok), vb16 = __float2bfloat16_rn(vx[j] * inv);
         if (pg >= 0) { kdst[j] = kb16; kdst[v_off + j] = vb16; }
         qs[e0 + j] = qf;
@@ -820,7 +831,8 @@ __device__ void stage_tile_argmax(const MegaArgs& a, MegaSmem* sm, int wtid) {
             for (int c = ts.y + 2; c <= ts.z; ++c) lg += __ldcg(a.partial + (size_t)c * cta_stride + off);
             lg *= sm->inv_s[r];
             if (a.dump_logits) a.dump_logits[(size_t)r * a.V + v] = lg;
-            if (!(a.st.eos_at[r] > 0 && v == a.eos_id)) key = float_order_key(lg);
+            if (!(a.st.eos_at[r] > 0 && v == a.eos_id))
+              key = float_order_key(decision_value(lg, a.sample, v, a.st.gen[r] + 1, a.st.row_key[r]));
           }
           const uint32_t best = __reduce_max_sync(0xffffffffu, key);
           const uint32_t who = __ballot_sync(0xffffffffu, key == best);
@@ -872,6 +884,7 @@ __device__ void stage_final(const MegaArgs& a, int wtid) {
         const int cap = a.st.scalars[0];
         const int gidx = a.st.gen[r] + 1;
         tok = (bi == 0x7fffffff) ? 0 : bi;
+        if (a.dump_choice) a.dump_choice[r] = tok;
         if (a.st.eos_at[r] > 0 && gidx == a.st.eos_at[r]) tok = a.eos_id;
         if (a.forced) tok = a.forced[r];
         a.st.out_tokens[(size_t)r * a.st.max_new + (gidx - 1)] = tok;
@@ -948,7 +961,7 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
         for (long long it = it0; it < it1; ++it, ++gi) {
           const int stage = gi % S;
           if (gi >= S) {
-            ok = mega_wait(smem_u32(&sm->empty[stage]), (uint32_t)(((gi / S) & 1) ^ 1), sm, a.status, kStatusProducerTimeout);
+            ok = mega_wait(smem_u32(&sm->empty[stage]), (uint32_t)(((gi / S) & 1) ^ 1), sm, a.status, kStatusProducerTimeout, a.wait_limit);
             if (!ok) break;
           }
           const uint32_t full = smem_u32(&sm->full[stage]);
@@ -979,7 +992,7 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
           while (sm->act_epoch <= gm) {
             __nanosleep(20);
             if (sm->abort) { ok = false; break; }
-            if (clock64() - t0 > 4000000000LL) {
+            if (clock64() - t0 > a.wait_limit) {
               atomicCAS(a.status, 0u, (uint32_t)kStatusFlagTimeout);
               sm->abort = 1;
               ok = false;
@@ -997,7 +1010,7 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
           while (sm->w_issued <= gi) {
             __nanosleep(40);
             if (sm->abort) { ok = false; break; }
-            if (clock64() - t0 > 4000000000LL) {
+            if (clock64() - t0 > a.wait_limit) {
               atomicCAS(a.status, 0u, (uint32_t)kStatusFlagTimeout);
               sm->abort = 1;
               ok = false;
@@ -1030,14 +1043,14 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
           if (seg_end > it1) seg_end = it1;
           const int buf = seg % acc_bufs;
           ok = mega_wait(smem_u32(&sm->acc_empty[buf]), (uint32_t)(((seg / acc_bufs) & 1) ^ 1), sm, a.status,
-                         kStatusMmaTimeout);
+                         kStatusMmaTimeout, a.wait_limit);
           if (!ok) break;
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + (uint32_t)(buf * kTileN);
           bool first = true;
           for (; it < seg_end; ++it, ++gi) {
             const int stage = gi % S;
-            ok = mega_wait(smem_u32(&sm->full[stage]), (uint32_t)((gi / S) & 1), sm, a.status, kStatusMmaTimeout);
+            ok = mega_wait(smem_u32(&sm->full[stage]), (uint32_t)((gi / S) & 1), sm, a.status, kStatusMmaTimeout, a.wait_limit);
             if (!ok) break;
             tc_fence_after();
             const uint64_t dw = smem_desc_sw128(w0 + (uint32_t)stage * kBlockBytes);
@@ -1093,7 +1106,7 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
         if (seg_end > it1) seg_end = it1;
         const int buf = seg % acc_bufs;
         ok = mega_wait(smem_u32(&sm->acc_full[buf]), (uint32_t)((seg / acc_bufs) & 1), sm, a.status,
-                       kStatusEpilogueTimeout);
+                       kStatusEpilogueTimeout, a.wait_limit);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
@@ -1156,6 +1169,17 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// Self-test of the bounded grid-wide wait, with nothing else in flight (no bulk copies, no tensor-core work): every
+// CTA arrives on the counter and then waits for one arrival more than the grid can deliver.  The wait must run out
+// after `limit` cycles, record kStatusGridBarrierTimeout and let the kernel end normally.
+__global__ void __launch_bounds__(32)
+grid_wait_selftest_kernel(unsigned long long* ctr, unsigned long long base, long long limit, uint32_t* status) {
+  if (threadIdx.x == 0) {
+    const unsigned long long target = base + (unsigned long long)gridDim.x + 1ULL;
+    if (!arrive_and_poll(ctr, target, limit, nullptr)) atomicCAS(status, 0u, (uint32_t)kStatusGridBarrierTimeout);
   }
 }
 

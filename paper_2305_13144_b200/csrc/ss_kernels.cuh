@@ -28,7 +28,7 @@ struct RowState {
   int32_t* active;       // 1 while the row is generating
   int32_t* finished;     // 1 once EOS was emitted
   int32_t* eos_at;       // 0 = natural EOS, t >= 1 = forced EOS at generated index t
-  int32_t* choice;       // argmax of the current step
+  int32_t* row_key;      // the row's key in the sampling counter (its query id inside a group)
   int32_t* out_tokens;   // [max_batch][max_new]
   int32_t* block_table;  // [max_batch][max_pages]
   int32_t* scalars;      // [0] = cap, [1] = n_active
@@ -128,10 +128,44 @@ __device__ __forceinline__ uint32_t float_order_key(float f) {      // monotone 
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
+// ---- sampling at a temperature (Sec. 4.2 generates at T = 0.5) ------------------------------------------
+// A draw from softmax(logits / T) is taken as argmax_v(logit_v / T + g_v) with Gumbel noise g_v = -log(-log(u_v)):
+// every u_v comes from the counter-based generator Philox4x32-10 (Salmon et al., SC'11) at counter
+// (vocabulary id, index of the generated token, row key, 0) and key (seed), so the arg-max machinery -- per
+// tile, then over tiles, in any order -- yields the same token as a sequential draw would.
+struct SampleCfg {
+  float inv_temp;        // 1 / T, or 0 for greedy decoding
+  uint32_t seed_lo, seed_hi;
+};
+
+__device__ __forceinline__ uint32_t philox4x32_10_word0(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0,
+                                                        uint32_t k1) {
+  constexpr uint32_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u, W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint32_t hi0 = __umulhi(M0, c0), lo0 = M0 * c0;
+    const uint32_t hi1 = __umulhi(M1, c2), lo1 = M1 * c2;
+    c0 = hi1 ^ c1 ^ k0;
+    c1 = lo1;
+    c2 = hi0 ^ c3 ^ k1;
+    c3 = lo0;
+    k0 += W0;
+    k1 += W1;
+  }
+  return c0;
+}
+// The value whose arg-max decides the token: the logit itself (greedy) or logit / T + Gumbel noise.
+__device__ __forceinline__ float decision_value(float logit, const SampleCfg& sc, int v, int gen_index, int row_key) {
+  if (sc.inv_temp == 0.f) return logit;
+  const uint32_t w = philox4x32_10_word0((uint32_t)v, (uint32_t)gen_index, (uint32_t)row_key, 0u, sc.seed_lo, sc.seed_hi);
+  const float u = ((float)(w >> 9) + 0.5f) * (1.0f / 8388608.0f);      // 24 significant bits, never 0 or 1
+  return fmaf(logit, sc.inv_temp, -logf(-logf(u)));
+}
+
 __global__ void __launch_bounds__(128)
 lmhead_tile_argmax_kernel(const float* __restrict__ partial, SplitInfo sp, RowState st, float* __restrict__ dump_logits,
                           float* __restrict__ tile_val, int32_t* __restrict__ tile_idx, int B, int vocab, int n_tiles,
-                          int eos_id) {
+                          int eos_id, SampleCfg sc) {
   __shared__ uint32_t s_key[4][kMaxBatch];
   __shared__ int s_id[4][kMaxBatch];
   pdl_launch_dependents();
@@ -144,7 +178,8 @@ lmhead_tile_argmax_kernel(const float* __restrict__ partial, SplitInfo sp, RowSt
       if (v < vocab) {
         const float lg = sum_partials(partial, sp, v, r);
         if (dump_logits) dump_logits[(size_t)r * vocab + v] = lg;
-        if (!(st.eos_at[r] > 0 && v == eos_id)) key = float_order_key(lg);
+        if (!(st.eos_at[r] > 0 && v == eos_id))
+          key = float_order_key(decision_value(lg, sc, v, st.gen[r] + 1, st.row_key[r]));
       }
       const uint32_t best = __reduce_max_sync(0xffffffffu, key);
       const uint32_t who = __ballot_sync(0xffffffffu, key == best);
@@ -173,8 +208,8 @@ lmhead_tile_argmax_kernel(const float* __restrict__ partial, SplitInfo sp, RowSt
 // by the host) and this is generated token 1; otherwise the fed token becomes part of the cache.
 __global__ void __launch_bounds__(1024)
 bookkeeping_kernel(RowState st, const float* __restrict__ tile_val, const int32_t* __restrict__ tile_idx, int n_tiles,
-                   const int32_t* __restrict__ forced, int32_t* __restrict__ next_tokens, int B, int eos_id,
-                   int is_prefill) {
+                   const int32_t* __restrict__ forced, int32_t* __restrict__ next_tokens, int32_t* __restrict__ dump_choice,
+                   int B, int eos_id, int is_prefill) {
   __shared__ int s_still;
   pdl_launch_dependents();
   pdl_wait();
@@ -203,6 +238,7 @@ bookkeeping_kernel(RowState st, const float* __restrict__ tile_val, const int32_
         const int cap = st.scalars[0];
         const int gidx = st.gen[r] + 1;               // 1-based index of the token being emitted
         tok = (bi == 0x7fffffff) ? 0 : bi;
+        if (dump_choice) dump_choice[r] = tok;
         if (st.eos_at[r] > 0 && gidx == st.eos_at[r]) tok = eos_id;
         if (forced) tok = forced[r];
         st.out_tokens[(size_t)r * st.max_new + (gidx - 1)] = tok;

@@ -67,11 +67,16 @@ noalloc_rmsnorm_kernel(const float* __restrict__ h, const __nv_bfloat16* __restr
     x[(size_t)r * d + i] = __float2bfloat16_rn(h[(size_t)r * d + i] * inv * __bfloat162float(g[i]));
 }
 
-// logits[r][v] = sum of the partials of output row v for token r, in CTA order.
+// logits[r][v] = sum of the partials of output row v for token r, in CTA order.  If a bounded wait of the
+// projection gave up (status word non-zero) the partials are not all there: the whole output becomes NaN,
+// which is how this call, having already returned, reports the failure.
 __global__ void __launch_bounds__(256)
-noalloc_reduce_kernel(const float* __restrict__ partial, SplitInfo sp, float* __restrict__ logits, int V) {
+noalloc_reduce_kernel(const float* __restrict__ partial, SplitInfo sp, float* __restrict__ logits, int V,
+                      const uint32_t* __restrict__ status) {
   const int r = blockIdx.y, v = blockIdx.x * blockDim.x + threadIdx.x;
-  if (v < V) logits[(size_t)r * V + v] = sum_partials_derived(partial, sp, v, r);
+  if (v >= V) return;
+  const bool failed = *status != 0u;
+  logits[(size_t)r * V + v] = failed ? __int_as_float(0x7fc00000) : sum_partials_derived(partial, sp, v, r);
 }
 
 int setup_device(int dev, DeviceSetup** out) {
@@ -94,7 +99,7 @@ int setup_device(int dev, DeviceSetup** out) {
       g_encode = (EncodeTiledFn)fn;
     }
     s.scratch = (unsigned char*)p;
-    s.n_sm = n < 148 ? n : 148;
+    s.n_sm = n;
     s.ready = true;
   }
   *out = &s;
@@ -121,6 +126,7 @@ extern "C" int ss_logits_noalloc(const float* hidden, const void* norm_gain, con
   if (n_rows > kNoAllocMaxRows || d_model > kNoAllocMaxD) return SS_ERR_CAPACITY;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return SS_ERR_CUDA;
+  (void)cudaGetLastError();   // an error left behind by the caller's earlier work is not this call's
   DeviceSetup* s = nullptr;
   int rc = setup_device(dev, &s);
   if (rc) return rc;
@@ -166,6 +172,6 @@ extern "C" int ss_logits_noalloc(const float* hidden, const void* norm_gain, con
   gemm_wx_kernel<<<dim3(1, p.gridx), kGemmThreads, p.smem_bytes, st>>>(mw, mx, a);
   SplitInfo sp;
   sp.gridx = p.gridx; sp.kb = p.kb; sp.max_seg = p.max_seg; sp.NT = p.NT; sp.total = total; sp.tiles = nullptr;
-  noalloc_reduce_kernel<<<dim3((vocab + 255) / 256, n_rows), 256, 0, st>>>(partial, sp, logits, vocab);
+  noalloc_reduce_kernel<<<dim3((vocab + 255) / 256, n_rows), 256, 0, st>>>(partial, sp, logits, vocab, status);
   return cudaGetLastError() == cudaSuccess ? SS_OK : SS_ERR_CUDA;
 }

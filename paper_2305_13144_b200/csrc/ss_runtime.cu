@@ -1,6 +1,6 @@
 // Host runtime behind the C ABI: context, arena carve-up, weight repacking, key/value page
-// allocator, kernel sequencing (prompt pass, decode step, CUDA-graph replay) and the group loop
-// of Sec. 4.1 (micro-batches, caps, failure collection and recomputation).
+// allocator, kernel sequencing (prompt pass, decode steps) and the group loop of Sec. 4.1
+// (micro-batches, caps, failure collection and recomputation).
 #include <algorithm>
 #include <cmath>
 #include <cstdio>
@@ -124,8 +124,11 @@ struct ss_ctx {
   ss_model_cfg m;
   ss_runtime_cfg rt;
   cudaStream_t stream;
-  int n_sm = 148;
+  int n_sm = 0;
   bool use_pdl = true;
+  bool trace_on = false;
+  long long wait_limit = 4000000000LL;   // SM cycles (about 2 s) any wait inside a kernel may last
+  int clock_khz = 1965000;
   int last_cuda = 0;
   int64_t launches = 0;
   EncodeTiledFn encode = nullptr;
@@ -181,6 +184,9 @@ struct ss_ctx {
   bool in_batch = false;
   std::vector<int32_t> prompt_len;
   int32_t* pinned = nullptr;     // [0] n_active, [1] status
+  // ---- sampling (greedy while inv_temp == 0)
+  SampleCfg sample{0.f, 0u, 0u};
+  std::vector<int32_t> next_row_keys;   // keys of the next batch's rows; empty = 0, 1, 2, ...
 };
 
 namespace {
@@ -370,6 +376,8 @@ void layout(const ss_model_cfg& m, const ss_runtime_cfg& rt, int n_sm, Offsets& 
   o.total = a.total;
 }
 
+// SMs of the current device; 148 (a B200) when no device can be asked, e.g. when sizing an arena on a host
+// without a GPU.
 int query_sms() {
   int dev = 0, n = 148;
   if (cudaGetDevice(&dev) == cudaSuccess) {
@@ -413,6 +421,17 @@ int weight_slot(const ss_ctx* c, const std::string& name, WeightSlot* out) {
     if (k == "w_down") return tiled(w.wdown, d, F, base + 8, 0);
   }
   return SS_ERR_ARG;
+}
+
+// A non-zero status word: the step that set it was abandoned half way.  The error is reported once; the word
+// and the grid-barrier counter (left in an unknown state by the abort) are cleared so that the context can
+// start a new batch.
+int report_device_status(ss_ctx* c, uint32_t word) {
+  cudaMemsetAsync(c->grid_ctr, 0, 8, c->stream);
+  cudaMemsetAsync(c->status, 0, 4, c->stream);
+  cudaStreamSynchronize(c->stream);
+  c->grid_epochs = 0;
+  return word == (uint32_t)kStatusBadPage ? SS_ERR_STATE : SS_ERR_DEVICE_TIMEOUT;
 }
 
 double weight_bytes_per_step(const ss_model_cfg& m) {
@@ -466,10 +485,13 @@ int enqueue_decode_step(ss_ctx* c, const ss_step_opts* opts, int32_t* next_token
   a.next_tokens = next_tokens;
   a.dump_logits = opts ? opts->dump_logits : nullptr;
   a.dump_hidden = opts ? opts->dump_hidden : nullptr;
+  a.dump_choice = opts ? opts->dump_choice : nullptr;
+  a.sample = c->sample;
   a.grid_ctr = c->grid_ctr;
   a.grid_base = c->grid_epochs * (unsigned long long)c->n_sm;
   a.status = c->status;
-  a.trace = c->trace;
+  a.trace = c->trace_on ? c->trace : nullptr;
+  a.wait_limit = c->wait_limit;
   void* args[4] = {(void*)mx, (void*)mo, (void*)ma, (void*)&a};
   const void* fn = m.head_dim == 128 ? (const void*)decode_step_mega_kernel<128> : (const void*)decode_step_mega_kernel<64>;
   SS_CUDA(c, cudaLaunchCooperativeKernel(fn, dim3(c->n_sm), dim3(kMegaThreads), args, smem, c->stream));
@@ -543,7 +565,7 @@ int ss_arena_bytes(const ss_model_cfg* model, const ss_runtime_cfg* rt, size_t* 
   if (rc) return rc;
   if (!out_bytes) return SS_ERR_ARG;
   Offsets o;
-  layout(*model, *rt, 148, o);          // sized for the largest grid the kernels use
+  layout(*model, *rt, query_sms(), o);  // the split tables and partial sums are sized by the SM count
   *out_bytes = o.total;
   return SS_OK;
 }
@@ -556,14 +578,19 @@ int ss_create(const ss_model_cfg* model, const ss_runtime_cfg* rt, void* dev_are
   int ndev = 0;
   if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) return SS_ERR_CUDA;
   Offsets o;
-  layout(*model, *rt, 148, o);
+  const int n_sm = query_sms();
+  layout(*model, *rt, n_sm, o);
   if (arena_bytes < o.total) return SS_ERR_CAPACITY;
   ss_ctx* c = new ss_ctx();
   c->m = *model;
   c->rt = *rt;
   c->stream = (cudaStream_t)stream;
-  c->n_sm = std::min(148, query_sms());
-  c->use_pdl = getenv("SS_NO_PDL") == nullptr;
+  c->n_sm = n_sm;
+  {
+    int dev = 0, khz = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetAttribute(&khz, cudaDevAttrClockRate, dev) == cudaSuccess && khz > 0)
+      c->clock_khz = khz;
+  }
   void* fn = nullptr;
   cudaDriverEntryPointQueryResult qr;
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qr) != cudaSuccess || !fn) {
@@ -604,7 +631,7 @@ int ss_create(const ss_model_cfg* model, const ss_runtime_cfg* rt, void* dev_are
   c->st.active = rows + 3 * kMaxBatch;
   c->st.finished = rows + 4 * kMaxBatch;
   c->st.eos_at = rows + 5 * kMaxBatch;
-  c->st.choice = rows + 6 * kMaxBatch;
+  c->st.row_key = rows + 6 * kMaxBatch;
   c->st.scalars = rows + 7 * kMaxBatch;
   c->st.block_table = (int32_t*)(A + o.block_table);
   c->st.out_tokens = (int32_t*)(A + o.out_tokens);
@@ -797,7 +824,9 @@ int ss_prefill(ss_ctx* c, const int32_t* tokens, const int32_t* cu, int32_t B, c
     rows[0 * kMaxBatch + r] = c->prompt_len[r];   // ctx_len after the prompt pass
     rows[3 * kMaxBatch + r] = 1;                  // active
     rows[5 * kMaxBatch + r] = eos_at ? eos_at[r] : 0;
+    rows[6 * kMaxBatch + r] = r < (int)c->next_row_keys.size() ? c->next_row_keys[r] : r;
   }
+  c->next_row_keys.clear();
   rows[7 * kMaxBatch + 0] = cap;
   rows[7 * kMaxBatch + 1] = B;
   int rc = SS_OK;
@@ -847,10 +876,10 @@ int ss_prefill(ss_ctx* c, const int32_t* tokens, const int32_t* cu, int32_t B, c
   if ((rc = run_gemm(c, c->lm_head, *mx, p_lm, kGemmPartial, B, nullptr, nullptr, 0))) return bail(rc);
   SS_CUDA_B(launch(c, lmhead_tile_argmax_kernel, dim3(c->n_tiles_lm), dim3(128), 0, (const float*)c->partial,
                    split_of(p_lm, c->tbl_lm_prompt), c->st, opts ? opts->dump_logits : (float*)nullptr, c->tile_val,
-                   c->tile_idx, B, m.vocab, c->n_tiles_lm, m.eos_id));
+                   c->tile_idx, B, m.vocab, c->n_tiles_lm, m.eos_id, c->sample));
   SS_CUDA_B(launch(c, bookkeeping_kernel, dim3(1), dim3(1024), 0, c->st, (const float*)c->tile_val,
                    (const int32_t*)c->tile_idx, c->n_tiles_lm, opts ? opts->forced_tokens : (const int32_t*)nullptr,
-                   first_tokens, B, m.eos_id, 1));
+                   first_tokens, opts ? opts->dump_choice : (int32_t*)nullptr, B, m.eos_id, 1));
 #undef SS_CUDA_B
   return SS_OK;
 }
@@ -886,13 +915,7 @@ int ss_read_batch(ss_ctx* c, int32_t* out_tokens, int32_t stride, int32_t* out_l
   SS_CUDA(c, cudaMemcpyAsync(fin.data(), c->st.finished, (size_t)B * 4, cudaMemcpyDeviceToHost, c->stream));
   SS_CUDA(c, cudaMemcpyAsync(c->pinned + 1, c->status, 4, cudaMemcpyDeviceToHost, c->stream));
   SS_CUDA(c, cudaStreamSynchronize(c->stream));
-  if (c->pinned[1] != 0) {
-    // an aborted step leaves the grid-barrier counter in an unknown state
-    cudaMemsetAsync(c->grid_ctr, 0, 8, c->stream);
-    cudaStreamSynchronize(c->stream);
-    c->grid_epochs = 0;
-    return c->pinned[1] == (int32_t)kStatusBadPage ? SS_ERR_STATE : SS_ERR_DEVICE_TIMEOUT;
-  }
+  if (c->pinned[1] != 0) return report_device_status(c, (uint32_t)c->pinned[1]);
   for (int r = 0; r < B; ++r) {
     if (out_tokens && gen[r] > stride) return SS_ERR_CAPACITY;
     out_len[r] = gen[r];
@@ -926,8 +949,55 @@ int ss_last_device_status(ss_ctx* c, uint32_t* out) {
   return SS_OK;
 }
 
+int ss_set_sampling(ss_ctx* c, float temperature, uint64_t seed) {
+  if (!c || !(temperature >= 0.f) || !std::isfinite(temperature)) return SS_ERR_ARG;
+  c->sample.inv_temp = temperature > 0.f ? 1.f / temperature : 0.f;
+  c->sample.seed_lo = (uint32_t)(seed & 0xffffffffu);
+  c->sample.seed_hi = (uint32_t)(seed >> 32);
+  return SS_OK;
+}
+
+int ss_set_row_keys(ss_ctx* c, const int32_t* keys, int32_t n) {
+  if (!c || n < 0 || n > kMaxBatch || (n > 0 && !keys)) return SS_ERR_ARG;
+  c->next_row_keys.assign(keys, keys + n);
+  return SS_OK;
+}
+
+int ss_set_wait_limit_ms(ss_ctx* c, int32_t ms) {
+  if (!c || ms < 1 || ms > 60000) return SS_ERR_ARG;
+  c->wait_limit = (long long)ms * c->clock_khz;
+  return SS_OK;
+}
+
+int ss_selftest_wait_timeout(ss_ctx* c, int32_t limit_us) {
+  if (!c || limit_us < 1 || limit_us > 1000000) return SS_ERR_ARG;
+  if (c->in_batch) return SS_ERR_STATE;
+  const long long limit = (long long)limit_us * c->clock_khz / 1000;
+  unsigned long long base = c->grid_epochs * (unsigned long long)c->n_sm;
+  unsigned long long* ctr = c->grid_ctr;
+  uint32_t* status = c->status;
+  void* args[4] = {(void*)&ctr, (void*)&base, (void*)&limit, (void*)&status};
+  SS_CUDA(c, cudaLaunchCooperativeKernel((const void*)grid_wait_selftest_kernel, dim3(c->n_sm), dim3(32), args, 0, c->stream));
+  c->launches++;
+  SS_CUDA(c, cudaMemcpyAsync(c->pinned + 1, c->status, 4, cudaMemcpyDeviceToHost, c->stream));
+  SS_CUDA(c, cudaStreamSynchronize(c->stream));
+  if (c->pinned[1] != 0) return report_device_status(c, (uint32_t)c->pinned[1]);
+  // the wait came through although an arrival was missing: the counter no longer matches the epochs
+  cudaMemsetAsync(c->grid_ctr, 0, 8, c->stream);
+  cudaStreamSynchronize(c->stream);
+  c->grid_epochs = 0;
+  return SS_OK;
+}
+
+int ss_set_trace(ss_ctx* c, int32_t on) {
+  if (!c) return SS_ERR_ARG;
+  c->trace_on = on != 0;
+  return SS_OK;
+}
+
 int ss_step_trace(ss_ctx* c, uint64_t* out, int32_t cap, int32_t* n) {
   if (!c || !out || !n) return SS_ERR_ARG;
+  if (!c->trace_on) return SS_ERR_STATE;
   *n = c->trace_len;
   if (cap < c->trace_len) return SS_ERR_CAPACITY;
   SS_CUDA(c, cudaMemcpyAsync(out, c->trace, (size_t)c->trace_len * 8, cudaMemcpyDeviceToHost, c->stream));
@@ -959,9 +1029,21 @@ int ss_run_group(ss_ctx* c, const ss_sched_cfg* cfg, const int32_t* prompt_token
   if ((rc = plan_first_pass(*cfg, plen.data(), pred_len, perm, n, ord, plan))) return rc;
   std::copy(ord.begin(), ord.end(), order);
 
-  cudaEvent_t ev[3];
-  for (auto& e : ev) SS_CUDA(c, cudaEventCreate(&e));
-  auto destroy_events = [&]() { for (auto& e : ev) cudaEventDestroy(e); };
+  cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};   // batch: start, prompt pass done, decode done; group: start, end
+  auto cleanup = [&](int code) {
+    for (auto& e : ev)
+      if (e) cudaEventDestroy(e);
+    if (c->in_batch) ss_release_batch(c);
+    return code;
+  };
+  // every CUDA failure below leaves through cleanup(): events destroyed, pages of a batch in flight returned
+#define SS_CUDA_G(expr)                                                          \
+  do {                                                                           \
+    cudaError_t _e = (expr);                                                     \
+    if (_e != cudaSuccess) { c->last_cuda = (int)_e; return cleanup(SS_ERR_CUDA); } \
+  } while (0)
+  for (auto& e : ev) SS_CUDA_G(cudaEventCreate(&e));
+  cudaEvent_t &g0 = ev[3], &g1 = ev[4];
 
   ss_group_stats gs{};
   const int64_t launches0 = c->launches;
@@ -974,17 +1056,7 @@ int ss_run_group(ss_ctx* c, const ss_sched_cfg* cfg, const int32_t* prompt_token
   size_t next_fail = 0;
   size_t bi = 0;
   const int B0 = cfg->base_batch;
-  cudaEvent_t g0, g1;
-  SS_CUDA(c, cudaEventCreate(&g0));
-  SS_CUDA(c, cudaEventCreate(&g1));
-  SS_CUDA(c, cudaEventRecord(g0, c->stream));
-  auto cleanup = [&](int code) {
-    destroy_events();
-    cudaEventDestroy(g0);
-    cudaEventDestroy(g1);
-    if (c->in_batch) ss_release_batch(c);
-    return code;
-  };
+  SS_CUDA_G(cudaEventRecord(g0, c->stream));
   for (;;) {
     ss_batch_desc b;
     const int32_t* rows_src;
@@ -1011,10 +1083,11 @@ int ss_run_group(ss_ctx* c, const ss_sched_cfg* cfg, const int32_t* prompt_token
       cu.push_back((int32_t)toks.size());
       if (eos_at) { eos_b.push_back(eos_at[q]); max_target = std::max(max_target, eos_at[q]); }
     }
-    SS_CUDA(c, cudaEventRecord(ev[0], c->stream));
+    c->next_row_keys.assign(rows_src, rows_src + B);      // a row's sampling key is its query id, in every pass
+    SS_CUDA_G(cudaEventRecord(ev[0], c->stream));
     rc = ss_prefill(c, toks.data(), cu.data(), B, eos_at ? eos_b.data() : nullptr, b.cap, nullptr, nullptr);
     if (rc) return cleanup(rc);
-    SS_CUDA(c, cudaEventRecord(ev[1], c->stream));
+    SS_CUDA_G(cudaEventRecord(ev[1], c->stream));
     if (eos_at) {
       // lengths are forced, so the number of steps is known: the longest target or the cap
       const int steps = std::min(b.cap, max_target);
@@ -1024,12 +1097,12 @@ int ss_run_group(ss_ctx* c, const ss_sched_cfg* cfg, const int32_t* prompt_token
       while (done < b.cap) {
         const int chunk = std::min(8, b.cap - done);
         if ((rc = ss_decode_steps(c, chunk, c->pinned))) return cleanup(rc);
-        SS_CUDA(c, cudaStreamSynchronize(c->stream));
+        SS_CUDA_G(cudaStreamSynchronize(c->stream));
         done += chunk;
         if (c->pinned[0] == 0) break;
       }
     }
-    SS_CUDA(c, cudaEventRecord(ev[2], c->stream));
+    SS_CUDA_G(cudaEventRecord(ev[2], c->stream));
     len_b.assign(B, 0);
     st_b.assign(B, 0);
     tok_b.assign((size_t)B * cfg->max_new_tokens, 0);
@@ -1067,8 +1140,9 @@ int ss_run_group(ss_ctx* c, const ss_sched_cfg* cfg, const int32_t* prompt_token
   }
   for (size_t i = 0; i < fail_rows.size(); ++i) order[n + i] = fail_rows[i];
   for (size_t i = fail_rows.size(); i < (size_t)n; ++i) order[n + i] = -1;
-  SS_CUDA(c, cudaEventRecord(g1, c->stream));
-  SS_CUDA(c, cudaEventSynchronize(g1));
+  SS_CUDA_G(cudaEventRecord(g1, c->stream));
+  SS_CUDA_G(cudaEventSynchronize(g1));
+#undef SS_CUDA_G
   cudaEventElapsedTime(&gs.total_ms, g0, g1);
   gs.n_batches = n_batches;
   gs.kernel_launches = c->launches - launches0;

@@ -9,68 +9,24 @@ import pytest
 from oracle import decoder as od
 from oracle import scheduler as osch
 from paper_2305_13144_b200 import synth
+from parity_util import (HIDDEN_TOL, LOGIT_TOL, assert_group_matches_simulation, engine, oracle_model,
+                         oracle_sched_cfg, teacher_forced)
 
 pytestmark = pytest.mark.gpu
 
-LOGIT_TOL = 2e-2
-HIDDEN_TOL = 1e-2
-
 
 def _oracle(shape, w):
-    return od.Decoder(w, n_layers=shape.n_layers, n_heads=shape.n_heads, head_dim=shape.head_dim,
-                      rms_eps=shape.rms_eps, rope_theta=shape.rope_theta, eos_id=shape.eos_id)
+    return oracle_model(shape, w)
 
 
-def _engine(shape, w, *, max_batch=16, max_ctx=128, max_prefill=512, max_new=64, kv_tokens=4096):
-    from paper_2305_13144_b200 import api
-    rt = api.runtime_cfg(max_batch, max_ctx, max_prefill, max_new, kv_tokens)
-    bits = {k: synth.to_bf16_bits(v) for k, v in w.items()}
-    return api.make_engine(shape, rt, bits)
+def _engine(shape, w, **kw):
+    return engine(shape, w, **kw)
 
 
 def _teacher_forced(shape, w, prompts, targets, cap, eng=None, **kw):
-    """Runs oracle and GPU side by side; returns worst relative logit error and hidden rel-L2."""
-    import torch
-    from paper_2305_13144_b200 import api
-    model = _oracle(shape, w)
-    B = len(prompts)
-    ref = [od.generate(model, p, cap, int(t), keep_logits=True, keep_hidden=True) for p, t in zip(prompts, targets)]
-    eng = eng or _engine(shape, w, **kw)
-    toks = np.concatenate([np.asarray(p, dtype=np.int32) for p in prompts])
-    cu = np.zeros(B + 1, dtype=np.int32)
-    cu[1:] = np.cumsum([len(p) for p in prompts])
-    dl = torch.zeros(B, shape.vocab, dtype=torch.float32, device="cuda")
-    dh = torch.zeros(B, shape.d_model, dtype=torch.float32, device="cuda")
-    nxt = torch.zeros(B, dtype=torch.int32, device="cuda")
-    steps = max(len(r["tokens"]) for r in ref)
-    worst_logit, worst_hidden = 0.0, 0.0
-    for t in range(steps):
-        alive = [r for r in range(B) if len(ref[r]["tokens"]) > t]
-        forced = torch.tensor([ref[r]["tokens"][t] if r in alive else shape.eos_id for r in range(B)],
-                              dtype=torch.int32, device="cuda")
-        if t == 0:
-            api.ss_prefill(eng, toks, cu, targets, cap, forced_tokens=forced, dump_logits=dl, dump_hidden=dh,
-                           first_tokens=nxt)
-        else:
-            api.ss_decode_step(eng, forced_tokens=forced, dump_logits=dl, dump_hidden=dh, next_tokens=nxt)
-        torch.cuda.synchronize()
-        assert api.ss_last_device_status(eng) == 0
-        gl, gh, gn = dl.cpu().numpy(), dh.cpu().numpy(), nxt.cpu().numpy()
-        for r in range(B):
-            if r in alive:
-                rl, rh = ref[r]["logits"][t], ref[r]["hidden"][t]
-                worst_logit = max(worst_logit, float(np.max(np.abs(gl[r] - rl)) / np.max(np.abs(rl))))
-                worst_hidden = max(worst_hidden, float(np.linalg.norm(gh[r] - rh) / np.linalg.norm(rh)))
-                assert gn[r] == ref[r]["tokens"][t]
-            else:
-                assert gn[r] == shape.eos_id           # finished rows report EOS and cost nothing
-    out, lens, status = api.ss_read_batch(eng, B, cap)
-    for r in range(B):
-        assert lens[r] == len(ref[r]["tokens"])
-        assert out[r, :lens[r]].tolist() == ref[r]["tokens"]
-        assert bool(status[r]) == ref[r]["finished"]
-    api.ss_release_batch(eng)
-    return worst_logit, worst_hidden
+    """Oracle and engine side by side (all rows followed); returns worst relative logit error and hidden rel-L2."""
+    el, eh, _ = teacher_forced(shape, w, prompts, targets, cap, eng, **kw)
+    return el, eh
 
 
 @pytest.mark.parametrize("n_layers", [0, 1, 2])
@@ -177,24 +133,10 @@ def test_run_group_log_is_bit_exact_with_scheduler_oracle():
             cfg = api.sched_cfg(bin_size=16, base_batch=8, max_new_tokens=64, vanilla=vanilla)
             perm = synth.make_permutation(g.n, seed) if vanilla else None
             res = api.ss_run_group(eng, cfg, g.prompt_tokens, g.prompt_off, g.pred_len, perm, g.true_len)
-            ocfg = osch.SchedCfg(bin_size=16, base_batch=8, max_new_tokens=64, vanilla=vanilla)
-            sim = osch.simulate(g.prompt_len, g.pred_len, g.true_len, ocfg, perm)
-            order = res["order"]
-            assert order[:g.n].tolist() == sim["order"]
-            nf = len(sim["failures"])
-            assert order[g.n:g.n + nf].tolist() == sim["failures"] and (order[g.n + nf:] == -1).all()
-            assert len(res["log"]) == len(sim["batches"])
-            for rec, ob in zip(res["log"], sim["batches"]):
-                rows = order[rec["first_row"]:rec["first_row"] + rec["n_rows"]].tolist()
-                assert rows == ob.rows and rec["cap"] == ob.cap and rec["is_recompute"] == int(ob.is_recompute)
-                assert rec["steps"] == ob.steps and rec["n_failed"] == len(ob.failed)
-            assert res["len"].tolist() == g.true_len.tolist()              # every row finally reaches its EOS
-            assert res["status"].tolist() == [1] * g.n
+            sim = osch.simulate(g.prompt_len, g.pred_len, g.true_len, oracle_sched_cfg(cfg), perm)
+            assert_group_matches_simulation(res, sim, g.n, g.true_len, shape.eos_id)
+            assert res["status"].tolist() == [1] * g.n                     # every row finally reaches its EOS
             st = res["stats"]
-            assert st["useful_tokens"] == sim["useful_tokens"] and st["row_steps"] == sim["row_steps"]
-            assert st["steps"] == sim["steps"] and st["n_failed"] == nf
-            for i in range(g.n):
-                assert res["tokens"][i, g.true_len[i] - 1] == shape.eos_id
             assert st["kernel_launches"] > 0
 
 
@@ -248,62 +190,6 @@ def test_wide_ffn_reads_tile_tables_from_global_memory():
     el, eh = _teacher_forced(shape, w, prompts, targets, cap=4, max_batch=16, max_ctx=64, max_prefill=256,
                              max_new=8, kv_tokens=1024)
     assert el <= LOGIT_TOL and eh <= HIDDEN_TOL, (el, eh)
-
-
-def test_7b_shape_two_layers_sampled_rows():
-    """The 7B shape (d 4096, 32 heads x 128, FFN 11008, vocab 32000) cut to two layers, batch 16 with the
-    benchmark's prompt lengths; the oracle follows the three rows with the shortest prompts through the
-    prompt pass and two decode steps; all rows run free, and a row is compared for as long as its tokens
-    agree with the oracle's (a disagreement is only accepted on a near-tie of the oracle's top two logits).
-
-    Hidden-state tolerance here is 2e-2, not the 1e-2 of the small configuration: with N(0, 0.02) weights at
-    d = 4096 the projections' outputs (std ~0.4) dwarf the embedding (std 0.02), so the residual stream's
-    relative error IS the relative error of the bf16 operand chain.  Re-running the oracle's own arithmetic
-    with nothing changed but a round-to-bf16 at the operands the GPU stores in bf16 (normalised input,
-    q/k/v, attention output, SwiGLU output) gives 1.1e-2 on this input, 1.35e-2 with the prompt pass's two
-    extra roundings (q/k/v and gate/up leave its GEMMs as bf16) -- the floor of the format, not of the kernels."""
-    import torch
-    from paper_2305_13144_b200 import api
-    shape = synth.LLAMA_7B.with_layers(2)
-    w = synth.make_weights(shape, seed=7)
-    g = synth.group_7b_batch16(seed=0)
-    B = g.n
-    rows = np.argsort(g.prompt_len)[:3].tolist()
-    model = od.Decoder(w, n_layers=2, n_heads=shape.n_heads, head_dim=shape.head_dim, rms_eps=shape.rms_eps,
-                       rope_theta=shape.rope_theta, eos_id=shape.eos_id, dtype=np.float64)
-    steps = 3
-    ref = {r: od.generate(model, g.prompt(r).tolist(), steps, steps + 5, keep_logits=True, keep_hidden=True) for r in rows}
-    del model
-    eng = api.make_engine(shape, api.runtime_cfg(16, 768, 4096, 512, 16 * 768),
-                          {k: synth.to_bf16_bits(v) for k, v in w.items()})
-    cu = np.zeros(B + 1, dtype=np.int32)
-    cu[1:] = np.cumsum(g.prompt_len)
-    dl = torch.zeros(B, shape.vocab, dtype=torch.float32, device="cuda")
-    dh = torch.zeros(B, shape.d_model, dtype=torch.float32, device="cuda")
-    nxt = torch.zeros(B, dtype=torch.int32, device="cuda")
-    worst_l = worst_h = 0.0
-    for t in range(steps):
-        if t == 0:
-            api.ss_prefill(eng, g.prompt_tokens, cu, np.full(B, steps + 5, dtype=np.int32), 512,
-                           dump_logits=dl, dump_hidden=dh, first_tokens=nxt)
-        else:
-            api.ss_decode_step(eng, dump_logits=dl, dump_hidden=dh, next_tokens=nxt)
-        torch.cuda.synchronize()
-        assert api.ss_last_device_status(eng) == 0
-        gl, gh, gn = dl.cpu().numpy(), dh.cpu().numpy(), nxt.cpu().numpy()
-        for r in rows:
-            rl, rh = ref[r]["logits"][t], ref[r]["hidden"][t]
-            worst_l = max(worst_l, float(np.max(np.abs(gl[r] - rl)) / np.max(np.abs(rl))))
-            worst_h = max(worst_h, float(np.linalg.norm(gh[r] - rh) / np.linalg.norm(rh)))
-            # free running: the argmax must agree unless the oracle's top two logits are within the tolerance
-            top2 = np.sort(rl)[-2:]
-            if top2[1] - top2[0] > 2 * LOGIT_TOL * np.max(np.abs(rl)):
-                assert gn[r] == ref[r]["tokens"][t]
-        if any(gn[r] != ref[r]["tokens"][t] for r in rows):
-            break                                    # histories diverged on a near-tie: nothing more to compare
-    assert t >= 1
-    assert worst_l <= LOGIT_TOL and worst_h <= 2e-2, (worst_l, worst_h)
-    api.ss_release_batch(eng)
 
 
 def test_full_size_7b_zero_output_projections_closed_form():
