@@ -328,6 +328,73 @@ def run_group_arms_7b(eng, api, kv_tok):
             "paper_context": "+86% samples/s on one A100-80G (Table 4), not comparable hardware"}
 
 
+def run_group_sweep(api, device):
+    """Throughput against group size (the paper's Fig. 3b: scheduling needs a group much larger than a micro-batch
+    and stops paying at 32): the 1024 queries at the 7B shape are processed in consecutive groups of G, each group
+    scheduled on its own (bins of 50 + FCR + variable batch size), against vanilla batching of the same groups."""
+    shape = synth.LLAMA_7B
+    kv_tok = 2 * shape.d_model * 2 * shape.n_layers
+    eng = make_engine(shape, api.runtime_cfg(256, 768, 16384, 512, int(120e9 // kv_tok)), seed=1234, device=device)
+    g = synth.group_7b_1024(seed=0)
+    perm = synth.make_permutation(g.n, 0)
+    points = []
+    for G in (32, 64, 128, 256, 512, 1024):
+        tot = {"vanilla": [0.0, 0], "scheduled": [0.0, 0]}
+        fails = 0
+        for lo in range(0, g.n, G):
+            ids = np.arange(lo, lo + G)
+            off = np.zeros(G + 1, dtype=np.int64)
+            off[1:] = np.cumsum(g.prompt_len[ids])
+            sub = synth.Group(np.concatenate([g.prompt(i) for i in ids]), off, g.prompt_len[ids], g.true_len[ids],
+                              g.pred_len[ids], g.max_new)
+            for name, cfg, pm in (("vanilla", api.sched_cfg(vanilla=True), np.argsort(perm[ids]).astype(np.int32)),
+                                  ("scheduled", api.sched_cfg(use_vbs=True, kv_budget_bytes=int(120e9),
+                                                              kv_bytes_per_token=kv_tok), None)):
+                r = run_group_arm(eng, api, sub, cfg, pm)
+                tot[name][0] += r["device_s"]
+                tot[name][1] += int(sub.true_len.sum())
+                if name == "scheduled":
+                    fails += int(round(r["failure_ratio"] * G))
+        v, sc = tot["vanilla"][1] / tot["vanilla"][0], tot["scheduled"][1] / tot["scheduled"][0]
+        points.append({"group_size": G, "vanilla_tokens_per_s": round(v, 1), "scheduled_tokens_per_s": round(sc, 1),
+                       "gain_vs_vanilla": round(sc / v, 3), "failure_ratio": round(fails / g.n, 3)})
+    return {"metric": METRIC, "unit": "tokens/s", "n_gpus": 1, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": "llama7b-shape bf16, 1024 queries in consecutive groups of G; FCR + VBS vs vanilla"},
+            "value": points[-1]["scheduled_tokens_per_s"], "points": points,
+            "paper_context": "Fig. 3b: throughput grows with the group size and scheduling fails at 32 (one A100-80G)"}
+
+
+def run_group_dispatch(api, device, rank, world, dist):
+    """Configuration 4's group dealt to `world` replicas (paper Sec. 1: micro-batches of different perceived
+    lengths go to different GPUs): one schedule, batches dealt longest estimated cost first, failures requeued
+    from a shared list; whole-job tokens/s = useful tokens / slowest replica's device time."""
+    from paper_2305_13144_b200.replicas import run_group_replicas
+    shape = synth.LLAMA_7B
+    kv_tok = 2 * shape.d_model * 2 * shape.n_layers
+    eng = make_engine(shape, api.runtime_cfg(256, 768, 16384, 512, int(120e9 // kv_tok)), seed=1234, device=device)
+    g = synth.group_7b_1024(seed=0)
+    cfg = api.sched_cfg(use_vbs=True, kv_budget_bytes=int(120e9), kv_bytes_per_token=kv_tok)
+
+    def gather(obj):
+        if world == 1:
+            return [obj]
+        box = [None] * world
+        dist.all_gather_object(box, obj)
+        return box
+
+    def run(order, batches):
+        return api.ss_run_batches(eng, cfg, g.prompt_tokens, g.prompt_off, g.true_len, order, batches)
+
+    res = run_group_replicas(api, cfg, g, None, rank=rank, world=world, run_batches=run, gather=gather, shape=shape)
+    assert res["len"].tolist() == g.true_len.tolist()
+    slowest = max(res["device_s"])
+    return {"metric": METRIC, "unit": "tokens/s", "n_gpus": world, "dtype": "bf16", "data": "synthetic",
+            "scaling": "strong", "higher_is_better": True,
+            "config": {"workload": "llama7b-shape bf16, 1024 queries, FCR + VBS, micro-batches dealt to replicas"},
+            "value": res["stats"]["useful_tokens"] / slowest, "device_s_per_replica": res["device_s"],
+            "batches": res["stats"]["n_batches"], "failure_ratio": res["stats"]["n_failed"] / g.n}
+
+
 def spawn_replicas(n: int) -> int:
     """`--gpus N` without a launcher: start one worker process per GPU (this script again, with the rank in the
     environment), pass rank 0's JSON line through, return the first non-zero exit code."""
@@ -485,6 +552,10 @@ def main():
                     help="instead of the batch-16 workload: cost of the length-perception pass against the scheduling gain")
     ap.add_argument("--sweep", action="store_true",
                     help="instead of the batch-16 workload: decode-step time over batch size and context (7B shape)")
+    ap.add_argument("--group-sweep", action="store_true",
+                    help="instead of the batch-16 workload: scheduled vs vanilla over the group size (7B shape)")
+    ap.add_argument("--group-dispatch", action="store_true",
+                    help="instead of the batch-16 workload: one 1024-query group dealt to the --gpus replicas")
     ap.add_argument("--layers", type=int, default=0, help="debug: truncate the model (invalidates the number)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
@@ -509,6 +580,17 @@ def main():
         os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
         dist.init_process_group("nccl", device_id=torch.device(device))
 
+    if args.group_dispatch:
+        out = run_group_dispatch(api, device, rank, world, dist)
+        if rank == 0:
+            print(json.dumps(out), flush=True)
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    if args.group_sweep:
+        if rank == 0:
+            print(json.dumps(run_group_sweep(api, device)), flush=True)
+        return
     if args.group_13b:
         if rank == 0:
             print(json.dumps(run_group_13b(api, device)), flush=True)

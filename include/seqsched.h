@@ -221,6 +221,29 @@ int ss_run_group(ss_ctx* ctx, const ss_sched_cfg* cfg, const int32_t* prompt_tok
                  int32_t* out_tokens, const int64_t* out_off, int32_t* out_len, uint8_t* out_status,
                  int32_t* order, ss_batch_log* log, int32_t log_cap, int32_t* n_log, ss_group_stats* stats);
 
+/* Runs a given list of micro-batches on this context, one after the other (the body of ss_run_group() without its
+ * scheduling): the unit of work when the batches of one schedule are dealt to several GPUs (Sec. 1: batches of
+ * different perceived lengths can go to different GPU nodes; each GPU holds a replica of the weights and no data
+ * crosses between GPUs while batches run).  Synchronous; all arguments host.
+ *   prompt_tokens / prompt_off [n+1], eos_at [n] or NULL   the whole group, as for ss_run_group
+ *   order [n_order], batches [n_batches]                    batch i = queries order[first_row .. first_row + n_rows)
+ *   out_tokens / out_off [n+1], out_len [n], out_status [n] written for the rows that ended here (not for failures)
+ *   fail_rows [n], n_fail                                   queries the cap cut (cap < max_new, no EOS), in batch
+ *                                                           and row order: the caller requeues them
+ *   log [log_cap], n_log, stats                             as for ss_run_group (stats may be NULL) */
+int ss_run_batches(ss_ctx* ctx, const ss_sched_cfg* cfg, const int32_t* prompt_tokens, const int64_t* prompt_off,
+                   const int32_t* eos_at, int32_t n, const int32_t* order, int32_t n_order, const ss_batch_desc* batches,
+                   int32_t n_batches, int32_t* out_tokens, const int64_t* out_off, int32_t* out_len, uint8_t* out_status,
+                   int32_t* fail_rows, int32_t* n_fail, ss_batch_log* log, int32_t log_cap, int32_t* n_log,
+                   ss_group_stats* stats);
+
+/* Deals micro-batches to n_gpus replicas (host only, pure).  The paper only proposes the hand-out (Sec. 1); the
+ * rule here: estimated cost of a batch = cap * (weight_bytes + rows * (mean prompt length + cap / 2) *
+ * kv_bytes_per_token) in integer arithmetic; batches in order of decreasing cost (ties: lower index) each go to the
+ * replica with the smallest total so far (ties: lowest replica).  gpu_of: host int32 [n_batches] (output). */
+int ss_deal_batches(const ss_batch_desc* batches, int32_t n_batches, const int32_t* order, const int32_t* prompt_len,
+                    int64_t weight_bytes, int64_t kv_bytes_per_token, int32_t n_gpus, int32_t* gpu_of);
+
 /* Bytes a decode step must move (weights once, plus the cached keys/values of the active
  * rows, plus the entries written); host arithmetic on lengths the caller supplies:
  * ctx_len host [B] (tokens cached before the step), active host uint8 [B]. */

@@ -162,3 +162,22 @@ def simulate(prompt_len, pred_len, true_len, cfg: SchedCfg, perm=None) -> dict:
         "avg_len_weighted": rowsteps / sum(len(b.rows) for b in log) if log else 0.0,
         "failure_ratio": len(failures) / n if n else 0.0,
     }
+
+
+def deal(batches, prompt_len, weight_bytes: int, kv_bytes_per_token: int, n_gpus: int) -> list:
+    """Replica dispatch of a batch list (Sec. 1 proposes handing micro-batches of different perceived lengths
+    to different GPUs; the rule itself is this build's): cost of a batch = cap * (weight_bytes +
+    rows * (mean prompt + cap / 2) * kv_bytes_per_token), all in integers; batches in order of decreasing cost
+    (ties: lower index) each go to the replica with the smallest total so far (ties: lowest replica).
+    Returns the replica of every batch."""
+    cost = []
+    for b in batches:
+        tokens2 = 2 * sum(int(prompt_len[r]) for r in b.rows) + len(b.rows) * b.cap
+        cost.append(b.cap * (weight_bytes + tokens2 * kv_bytes_per_token // 2))
+    load = [0] * n_gpus
+    out = [0] * len(batches)
+    for i in sorted(range(len(batches)), key=lambda i: (-cost[i], i)):
+        g = min(range(n_gpus), key=lambda g: (load[g], g))
+        out[i] = g
+        load[g] += cost[i]
+    return out

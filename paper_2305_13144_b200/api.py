@@ -23,7 +23,7 @@ EXPORTS = [
     "ss_arena_bytes", "ss_create", "ss_destroy", "ss_load_weights", "ss_schedule", "ss_prefill",
     "ss_decode_step", "ss_decode_steps", "ss_read_batch", "ss_release_batch", "ss_run_group",
     "ss_step_model_bytes", "ss_strerror", "ss_last_device_status", "ss_last_cuda_error", "ss_kernel_launches",
-    "ss_logits_noalloc", "ss_step_trace", "ss_set_trace", "ss_set_sampling", "ss_set_row_keys", "ss_set_wait_limit_ms", "ss_selftest_wait_timeout",
+    "ss_logits_noalloc", "ss_step_trace", "ss_set_trace", "ss_set_sampling", "ss_set_row_keys", "ss_run_batches", "ss_deal_batches", "ss_set_wait_limit_ms", "ss_selftest_wait_timeout",
 ]
 
 
@@ -103,6 +103,10 @@ def lib() -> C.CDLL:
         L.ss_read_batch.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
         L.ss_release_batch.argtypes = [C.c_void_p]
         L.ss_run_group.argtypes = [C.c_void_p] * 7 + [C.c_int32] + [C.c_void_p] * 6 + [C.c_int32, C.c_void_p, C.c_void_p]
+        L.ss_run_batches.argtypes = [C.c_void_p] * 5 + [C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_int32] + \
+                                    [C.c_void_p] * 6 + [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
+        L.ss_deal_batches.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int32,
+                                      C.c_void_p]
         L.ss_step_model_bytes.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(C.c_double)]
         L.ss_last_device_status.argtypes = [C.c_void_p, C.POINTER(C.c_uint32)]
         L.ss_step_trace.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(C.c_int32)]
@@ -298,6 +302,47 @@ def ss_run_group(ctx: Ctx, cfg: ss_sched_cfg, prompt_tokens, prompt_off, pred_le
         "log": [{f: getattr(b, f) for f in fields} for b in log[:n_log.value]],
         "stats": {f[0]: getattr(stats, f[0]) for f in ss_group_stats._fields_},
     }
+
+
+def _descs(batches):
+    arr = (ss_batch_desc * max(len(batches), 1))()
+    for i, b in enumerate(batches):
+        arr[i] = ss_batch_desc(*[int(x) for x in b])
+    return arr
+
+
+def ss_run_batches(ctx: Ctx, cfg: ss_sched_cfg, prompt_tokens, prompt_off, eos_at, order, batches) -> dict:
+    """batches: list of (first_row, n_rows, cap, is_recompute) indexing `order`.  Returns tokens / len / status
+    arrays over the whole group (valid for the rows that ended here), the failed queries, the log and the stats."""
+    pt, po, ea = _np(prompt_tokens, np.int32), _np(prompt_off, np.int64), _np(eos_at, np.int32)
+    od = _np(order, np.int32)
+    n = int(po.shape[0]) - 1
+    mx = cfg.max_new_tokens
+    out_off = np.arange(n + 1, dtype=np.int64) * mx
+    out_tokens = np.zeros(max(n * mx, 1), dtype=np.int32)
+    out_len = np.zeros(max(n, 1), dtype=np.int32)
+    out_status = np.zeros(max(n, 1), dtype=np.uint8)
+    fail = np.zeros(max(n, 1), dtype=np.int32)
+    n_fail, n_log = C.c_int32(0), C.c_int32(0)
+    log = (ss_batch_log * max(len(batches), 1))()
+    stats = ss_group_stats()
+    _check(lib().ss_run_batches(ctx.handle, C.byref(cfg), _hp(pt), _hp(po), _hp(ea), n, _hp(od), int(od.shape[0]),
+                                _descs(batches), len(batches), _hp(out_tokens), _hp(out_off), _hp(out_len),
+                                _hp(out_status), _hp(fail), C.byref(n_fail), log, len(batches), C.byref(n_log),
+                                C.byref(stats)), "ss_run_batches", ctx)
+    fields = [f[0] for f in ss_batch_log._fields_]
+    return {"tokens": out_tokens.reshape(n, mx), "len": out_len[:n], "status": out_status[:n],
+            "failed": fail[:n_fail.value].tolist(),
+            "log": [{f: getattr(b, f) for f in fields} for b in log[:n_log.value]],
+            "stats": {f[0]: getattr(stats, f[0]) for f in ss_group_stats._fields_}}
+
+
+def ss_deal_batches(batches, order, prompt_len, weight_bytes: int, kv_bytes_per_token: int, n_gpus: int) -> list:
+    od, pl = _np(order, np.int32), _np(prompt_len, np.int32)
+    out = np.zeros(max(len(batches), 1), dtype=np.int32)
+    _check(lib().ss_deal_batches(_descs(batches), len(batches), _hp(od), _hp(pl), int(weight_bytes),
+                                 int(kv_bytes_per_token), int(n_gpus), _hp(out)), "ss_deal_batches")
+    return out[:len(batches)].tolist()
 
 
 def ss_step_model_bytes(ctx: Ctx, ctx_len, active=None) -> float:

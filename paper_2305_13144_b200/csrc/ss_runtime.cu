@@ -1008,28 +1008,18 @@ int ss_step_trace(ss_ctx* c, uint64_t* out, int32_t cap, int32_t* n) {
 int ss_last_cuda_error(const ss_ctx* c) { return c ? c->last_cuda : 0; }
 int64_t ss_kernel_launches(const ss_ctx* c) { return c ? c->launches : 0; }
 
-int ss_run_group(ss_ctx* c, const ss_sched_cfg* cfg, const int32_t* prompt_tokens, const int64_t* prompt_off,
-                 const int32_t* pred_len, const int32_t* perm, const int32_t* eos_at, int32_t n, int32_t* out_tokens,
-                 const int64_t* out_off, int32_t* out_len, uint8_t* out_status, int32_t* order, ss_batch_log* log,
-                 int32_t log_cap, int32_t* n_log, ss_group_stats* stats) {
-  if (!c || !cfg || n < 0 || !n_log) return SS_ERR_ARG;
-  if (n > 0 && (!prompt_tokens || !prompt_off || !pred_len || !out_tokens || !out_off || !out_len || !out_status || !order))
-    return SS_ERR_ARG;
-  int rc = validate_sched_cfg(cfg);
-  if (rc) return rc;
-  if (c->in_batch) return SS_ERR_STATE;
-  if (cfg->max_new_tokens > c->rt.max_new_tokens) return SS_ERR_CAPACITY;
-  for (int i = 0; i < n; ++i)
-    if (out_off[i + 1] - out_off[i] < cfg->max_new_tokens) return SS_ERR_CAPACITY;
+}  // extern "C"
 
-  std::vector<int32_t> plen(n);
-  for (int i = 0; i < n; ++i) plen[i] = (int32_t)(prompt_off[i + 1] - prompt_off[i]);
-  std::vector<int32_t> ord;
-  std::vector<ss_batch_desc> plan;
-  if ((rc = plan_first_pass(*cfg, plen.data(), pred_len, perm, n, ord, plan))) return rc;
-  std::copy(ord.begin(), ord.end(), order);
-
-  cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};   // batch: start, prompt pass done, decode done; group: start, end
+// Runs the micro-batches batches[0..n_batches) (rows: order[first_row .. first_row + n_rows)) one after the other:
+// prompt pass, decode until every row has finished or the cap, read back.  Rows the cap cut (cap < max_new, no EOS)
+// are appended to `fails`; the others get their final tokens, length and status.  Adds to `gs`, writes one log record
+// per batch from log[*n_log] on.
+static int run_batch_list(ss_ctx* c, const ss_sched_cfg* cfg, const int32_t* prompt_tokens, const int64_t* prompt_off,
+                          const int32_t* eos_at, const int32_t* order, const ss_batch_desc* batches, int32_t n_batches,
+                          int32_t* out_tokens, const int64_t* out_off, int32_t* out_len, uint8_t* out_status,
+                          std::vector<int32_t>& fails, ss_batch_log* log, int32_t log_cap, int32_t* n_log,
+                          ss_group_stats& gs) {
+  cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};       // batch start, prompt pass done, decode done
   auto cleanup = [&](int code) {
     for (auto& e : ev)
       if (e) cudaEventDestroy(e);
@@ -1043,36 +1033,15 @@ int ss_run_group(ss_ctx* c, const ss_sched_cfg* cfg, const int32_t* prompt_token
     if (_e != cudaSuccess) { c->last_cuda = (int)_e; return cleanup(SS_ERR_CUDA); } \
   } while (0)
   for (auto& e : ev) SS_CUDA_G(cudaEventCreate(&e));
-  cudaEvent_t &g0 = ev[3], &g1 = ev[4];
-
-  ss_group_stats gs{};
-  const int64_t launches0 = c->launches;
   const double W = weight_bytes_per_step(c->m), kvt = kv_bytes_per_token(c->m);
-  std::vector<int32_t> fail_rows;
-  std::vector<int32_t> toks, cu, eos_b, len_b;
+  std::vector<int32_t> toks, cu, eos_b, len_b, tok_b;
   std::vector<uint8_t> st_b;
-  std::vector<int32_t> tok_b;
-  int n_batches = 0;
-  size_t next_fail = 0;
-  size_t bi = 0;
-  const int B0 = cfg->base_batch;
-  SS_CUDA_G(cudaEventRecord(g0, c->stream));
-  for (;;) {
-    ss_batch_desc b;
-    const int32_t* rows_src;
-    if (bi < plan.size()) {
-      b = plan[bi++];
-      rows_src = ord.data() + b.first_row;
-    } else if (next_fail < fail_rows.size()) {
-      const int nr = (int)std::min<size_t>(B0, fail_rows.size() - next_fail);
-      b = {(int32_t)(n + next_fail), nr, cfg->max_new_tokens, 1};
-      rows_src = fail_rows.data() + next_fail;
-      next_fail += nr;
-    } else {
-      break;
-    }
+  int rc;
+  for (int32_t bi = 0; bi < n_batches; ++bi) {
+    const ss_batch_desc b = batches[bi];
+    const int32_t* rows_src = order + b.first_row;
     const int B = b.n_rows;
-    if (n_batches >= log_cap && log) return cleanup(SS_ERR_CAPACITY);
+    if (log && *n_log >= log_cap) return cleanup(SS_ERR_CAPACITY);
     toks.clear();
     cu.assign(1, 0);
     eos_b.clear();
@@ -1117,7 +1086,7 @@ int ss_run_group(ss_ctx* c, const ss_sched_cfg* cfg, const int32_t* prompt_token
       steps = std::max(steps, len_b[r]);
       const bool failed = !st_b[r] && b.cap < cfg->max_new_tokens;
       if (failed) {
-        fail_rows.push_back(q);
+        fails.push_back(q);
         ++n_failed;
       } else {
         out_len[q] = len_b[r];
@@ -1130,25 +1099,128 @@ int ss_run_group(ss_ctx* c, const ss_sched_cfg* cfg, const int32_t* prompt_token
       gs.model_bytes += kvt * (nr * (cu[r + 1] - cu[r]) + nr * (nr + 1) / 2.0);
     }
     gs.model_bytes += W * std::max(0, steps - 1);
-    if (log) log[n_batches] = {b.first_row, B, b.cap, b.is_recompute, steps, n_failed, pf, dc};
-    ++n_batches;
+    if (log) log[*n_log] = {b.first_row, B, b.cap, b.is_recompute, steps, n_failed, pf, dc};
+    ++*n_log;
+    gs.n_batches += 1;
     gs.steps += steps;
     gs.row_steps += (int64_t)B * steps;
     gs.prefill_ms += pf;
     gs.decode_ms += dc;
     gs.n_failed += n_failed;
   }
-  for (size_t i = 0; i < fail_rows.size(); ++i) order[n + i] = fail_rows[i];
-  for (size_t i = fail_rows.size(); i < (size_t)n; ++i) order[n + i] = -1;
-  SS_CUDA_G(cudaEventRecord(g1, c->stream));
-  SS_CUDA_G(cudaEventSynchronize(g1));
 #undef SS_CUDA_G
-  cudaEventElapsedTime(&gs.total_ms, g0, g1);
-  gs.n_batches = n_batches;
-  gs.kernel_launches = c->launches - launches0;
-  *n_log = n_batches;
-  if (stats) *stats = gs;
   return cleanup(SS_OK);
+}
+
+extern "C" {
+
+int ss_run_batches(ss_ctx* c, const ss_sched_cfg* cfg, const int32_t* prompt_tokens, const int64_t* prompt_off,
+                   const int32_t* eos_at, int32_t n, const int32_t* order, int32_t n_order, const ss_batch_desc* batches,
+                   int32_t n_batches, int32_t* out_tokens, const int64_t* out_off, int32_t* out_len, uint8_t* out_status,
+                   int32_t* fail_rows, int32_t* n_fail, ss_batch_log* log, int32_t log_cap, int32_t* n_log,
+                   ss_group_stats* stats) {
+  if (!c || !cfg || n < 0 || n_batches < 0 || n_order < 0 || !n_log || !n_fail) return SS_ERR_ARG;
+  if (n_batches > 0 && (!prompt_tokens || !prompt_off || !order || !batches || !out_tokens || !out_off || !out_len ||
+                        !out_status || !fail_rows))
+    return SS_ERR_ARG;
+  int rc = validate_sched_cfg(cfg);
+  if (rc) return rc;
+  if (c->in_batch) return SS_ERR_STATE;
+  if (cfg->max_new_tokens > c->rt.max_new_tokens) return SS_ERR_CAPACITY;
+  for (int32_t i = 0; i < n_batches; ++i) {
+    const ss_batch_desc& b = batches[i];
+    if (b.n_rows < 1 || b.first_row < 0 || (int64_t)b.first_row + b.n_rows > n_order || b.cap < 1 ||
+        b.cap > cfg->max_new_tokens)
+      return SS_ERR_ARG;
+    for (int r = 0; r < b.n_rows; ++r) {
+      const int32_t q = order[b.first_row + r];
+      if (q < 0 || q >= n) return SS_ERR_ARG;
+      if (out_off[q + 1] - out_off[q] < cfg->max_new_tokens) return SS_ERR_CAPACITY;
+    }
+  }
+  cudaEvent_t g0 = nullptr, g1 = nullptr;
+  if (cudaEventCreate(&g0) != cudaSuccess || cudaEventCreate(&g1) != cudaSuccess) {
+    if (g0) cudaEventDestroy(g0);
+    return SS_ERR_CUDA;
+  }
+  ss_group_stats gs{};
+  const int64_t launches0 = c->launches;
+  std::vector<int32_t> fails;
+  *n_log = 0;
+  cudaEventRecord(g0, c->stream);
+  rc = run_batch_list(c, cfg, prompt_tokens, prompt_off, eos_at, order, batches, n_batches, out_tokens, out_off,
+                      out_len, out_status, fails, log, log_cap, n_log, gs);
+  if (rc == SS_OK) {
+    cudaEventRecord(g1, c->stream);
+    if (cudaEventSynchronize(g1) != cudaSuccess) rc = SS_ERR_CUDA;
+    else cudaEventElapsedTime(&gs.total_ms, g0, g1);
+  }
+  cudaEventDestroy(g0);
+  cudaEventDestroy(g1);
+  if (rc) return rc;
+  std::copy(fails.begin(), fails.end(), fail_rows);
+  *n_fail = (int32_t)fails.size();
+  gs.kernel_launches = c->launches - launches0;
+  if (stats) *stats = gs;
+  return SS_OK;
+}
+
+int ss_run_group(ss_ctx* c, const ss_sched_cfg* cfg, const int32_t* prompt_tokens, const int64_t* prompt_off,
+                 const int32_t* pred_len, const int32_t* perm, const int32_t* eos_at, int32_t n, int32_t* out_tokens,
+                 const int64_t* out_off, int32_t* out_len, uint8_t* out_status, int32_t* order, ss_batch_log* log,
+                 int32_t log_cap, int32_t* n_log, ss_group_stats* stats) {
+  if (!c || !cfg || n < 0 || !n_log) return SS_ERR_ARG;
+  if (n > 0 && (!prompt_tokens || !prompt_off || !pred_len || !out_tokens || !out_off || !out_len || !out_status || !order))
+    return SS_ERR_ARG;
+  int rc = validate_sched_cfg(cfg);
+  if (rc) return rc;
+  if (c->in_batch) return SS_ERR_STATE;
+  if (cfg->max_new_tokens > c->rt.max_new_tokens) return SS_ERR_CAPACITY;
+  for (int i = 0; i < n; ++i)
+    if (out_off[i + 1] - out_off[i] < cfg->max_new_tokens) return SS_ERR_CAPACITY;
+
+  std::vector<int32_t> plen(n);
+  for (int i = 0; i < n; ++i) plen[i] = (int32_t)(prompt_off[i + 1] - prompt_off[i]);
+  std::vector<int32_t> ord;
+  std::vector<ss_batch_desc> plan;
+  if ((rc = plan_first_pass(*cfg, plen.data(), pred_len, perm, n, ord, plan))) return rc;
+
+  cudaEvent_t g0 = nullptr, g1 = nullptr;
+  if (cudaEventCreate(&g0) != cudaSuccess || cudaEventCreate(&g1) != cudaSuccess) {
+    if (g0) cudaEventDestroy(g0);
+    return SS_ERR_CUDA;
+  }
+  auto done = [&](int code) { cudaEventDestroy(g0); cudaEventDestroy(g1); return code; };
+  ss_group_stats gs{};
+  const int64_t launches0 = c->launches;
+  std::vector<int32_t> fails;
+  *n_log = 0;
+  cudaEventRecord(g0, c->stream);
+  // first pass
+  rc = run_batch_list(c, cfg, prompt_tokens, prompt_off, eos_at, ord.data(), plan.data(), (int32_t)plan.size(),
+                      out_tokens, out_off, out_len, out_status, fails, log, log_cap, n_log, gs);
+  if (rc) return done(rc);
+  // the rows the caps cut, in collection order, regenerated from their prompts in batches of B0 with cap = max_new
+  // (Sec. 4.1, failure collection and recomputation); they are listed behind the first-pass order
+  const size_t n_fail = fails.size();
+  ord.insert(ord.end(), fails.begin(), fails.end());
+  std::vector<ss_batch_desc> again;
+  for (size_t i = 0; i < n_fail; i += (size_t)cfg->base_batch)
+    again.push_back({(int32_t)(n + i), (int32_t)std::min<size_t>(cfg->base_batch, n_fail - i), cfg->max_new_tokens, 1});
+  std::vector<int32_t> fails2;
+  rc = run_batch_list(c, cfg, prompt_tokens, prompt_off, eos_at, ord.data(), again.data(), (int32_t)again.size(),
+                      out_tokens, out_off, out_len, out_status, fails2, log, log_cap, n_log, gs);
+  if (rc) return done(rc);
+  gs.n_failed = (int32_t)n_fail;
+  for (int i = 0; i < n; ++i) order[i] = ord[i];
+  for (size_t i = 0; i < n_fail; ++i) order[n + i] = fails[i];
+  for (size_t i = n_fail; i < (size_t)n; ++i) order[n + i] = -1;
+  cudaEventRecord(g1, c->stream);
+  if (cudaEventSynchronize(g1) != cudaSuccess) return done(SS_ERR_CUDA);
+  cudaEventElapsedTime(&gs.total_ms, g0, g1);
+  gs.kernel_launches = c->launches - launches0;
+  if (stats) *stats = gs;
+  return done(SS_OK);
 }
 
 }  // extern "C"

@@ -93,6 +93,40 @@ int plan_first_pass(const ss_sched_cfg& c, const int32_t* prompt_len, const int3
 
 }  // namespace ss
 
+// Replica dispatch (Sec. 1: micro-batches of different perceived lengths can be handed to different GPUs).
+// Estimated cost of a batch = its steps (the cap) times the bytes one decode step moves: the weights once plus, per
+// row, the cached keys and values at the batch's mean prompt length plus half the cap.  Batches are taken in order
+// of decreasing cost (equal costs: lower index first); each goes to the replica whose total is smallest so far
+// (equal totals: lowest replica).
+extern "C" int ss_deal_batches(const ss_batch_desc* batches, int32_t n_batches, const int32_t* order,
+                               const int32_t* prompt_len, int64_t weight_bytes, int64_t kv_bytes_per_token,
+                               int32_t n_gpus, int32_t* gpu_of) {
+  if (n_batches < 0 || n_gpus < 1 || weight_bytes < 0 || kv_bytes_per_token < 0) return SS_ERR_ARG;
+  if (n_batches > 0 && (!batches || !order || !prompt_len || !gpu_of)) return SS_ERR_ARG;
+  std::vector<int64_t> cost(n_batches);
+  for (int32_t i = 0; i < n_batches; ++i) {
+    const ss_batch_desc& b = batches[i];
+    if (b.n_rows < 1 || b.first_row < 0 || b.cap < 1) return SS_ERR_ARG;
+    int64_t prompt_sum = 0;
+    for (int32_t r = 0; r < b.n_rows; ++r) prompt_sum += prompt_len[order[b.first_row + r]];
+    // rows * (mean prompt + cap / 2) cached tokens, kept in integers: (2 * prompt_sum + rows * cap) / 2
+    const int64_t tokens2 = 2 * prompt_sum + (int64_t)b.n_rows * b.cap;
+    cost[i] = (int64_t)b.cap * (weight_bytes + tokens2 * kv_bytes_per_token / 2);
+  }
+  std::vector<int32_t> by_cost(n_batches);
+  for (int32_t i = 0; i < n_batches; ++i) by_cost[i] = i;
+  std::stable_sort(by_cost.begin(), by_cost.end(), [&](int32_t a, int32_t b) { return cost[a] > cost[b]; });
+  std::vector<int64_t> load(n_gpus, 0);
+  for (int32_t i : by_cost) {
+    int32_t best = 0;
+    for (int32_t g = 1; g < n_gpus; ++g)
+      if (load[g] < load[best]) best = g;
+    gpu_of[i] = best;
+    load[best] += cost[i];
+  }
+  return SS_OK;
+}
+
 extern "C" int ss_schedule(const ss_sched_cfg* cfg, const int32_t* prompt_len, const int32_t* pred_len,
                            const int32_t* perm, int32_t n, int32_t* order, ss_batch_desc* batches,
                            int32_t batch_cap, int32_t* n_batches) {
