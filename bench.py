@@ -230,6 +230,48 @@ def cpu_baseline_leg():
             "sample": f"{what}; {spent:.1f}s of CPU time; numpy on {cores} threads"}
 
 
+def run_cpu_extras():
+    """The oracle timed on the host cores beyond the default line's sample: configuration 1 end to end (the small
+    model, 32 queries: vanilla batching and sequence scheduling, every micro-batch and the recomputation batches
+    generated by the oracle decoder), and the scheduler oracle alone on the groups of configurations 3, 4 and 5."""
+    from oracle import decoder as od
+    from oracle import scheduler as osch
+    shape = synth.TINY
+    w = synth.make_weights(shape, seed=1234)
+    model = od.Decoder(w, n_layers=shape.n_layers, n_heads=shape.n_heads, head_dim=shape.head_dim,
+                       rms_eps=shape.rms_eps, rope_theta=shape.rope_theta, eos_id=shape.eos_id)
+    g = synth.group_tiny(seed=0)
+    out = {"cores": os.cpu_count(), "config1": {}, "scheduler_alone": {}}
+    for name, cfg, perm in (("vanilla", osch.SchedCfg(bin_size=16, base_batch=8, max_new_tokens=64, vanilla=True),
+                             synth.make_permutation(g.n, 0)),
+                            ("scheduled_fcr", osch.SchedCfg(bin_size=16, base_batch=8, max_new_tokens=64), None)):
+        sim = osch.simulate(g.prompt_len, g.pred_len, g.true_len, cfg, perm)
+        t0 = time.time()
+        for b in sim["batches"]:
+            res = od.run_micro_batch(model, [g.prompt(r).tolist() for r in b.rows], b.cap, [int(g.true_len[r]) for r in b.rows])
+            assert res["steps"] == b.steps
+        dt = time.time() - t0
+        out["config1"][name] = {"seconds": round(dt, 2), "tokens_per_s": round(sim["useful_tokens"] / dt, 1),
+                                "samples_per_s": round(g.n / dt, 2), "steps": sim["steps"], "batches": len(sim["batches"])}
+    out["config1"]["gain_vs_vanilla"] = round(out["config1"]["scheduled_fcr"]["tokens_per_s"] /
+                                              out["config1"]["vanilla"]["tokens_per_s"], 3)
+    kv7 = 2 * synth.LLAMA_7B.d_model * 2 * synth.LLAMA_7B.n_layers
+    kv13 = 2 * synth.LLAMA_13B.d_model * 2 * synth.LLAMA_13B.n_layers
+    cases = (("config3 (1024 queries, FCR, batch 16)", synth.group_7b_1024(0), osch.SchedCfg()),
+             ("config4 (1024 queries, FCR + VBS, 120 GB)", synth.group_7b_1024(0),
+              osch.SchedCfg(use_vbs=True, kv_budget_bytes=int(120e9), kv_bytes_per_token=kv7)),
+             ("config5 (512 queries, 13B shape, FCR + VBS)", synth.group_13b_512(0),
+              osch.SchedCfg(use_vbs=True, max_new_tokens=2048, kv_budget_bytes=int(120e9), kv_bytes_per_token=kv13)))
+    for name, grp, cfg in cases:
+        reps = 20
+        t0 = time.time()
+        for _ in range(reps):
+            sim = osch.simulate(grp.prompt_len, grp.pred_len, grp.true_len, cfg)
+        out["scheduler_alone"][name] = {"ms": round((time.time() - t0) / reps * 1e3, 2), "batches": len(sim["batches"]),
+                                        "steps": sim["steps"]}
+    return out
+
+
 def aggregate(tokens_local: float, seconds_local: float, dist):
     """Whole-job numbers from per-rank ones: tokens add up, time is the slowest rank's."""
     import torch
@@ -459,13 +501,17 @@ def run_perception(api, device):
     """What the length-perception pass costs against what scheduling gains (the paper's paragraph on the
     overhead of length prediction, Sec. 4.2): every query's prompt plus a 32-token instruction suffix is
     processed and 3 tokens are generated (the predicted number), in batches of 256, before the group is
-    scheduled; the predictions themselves are the synthetic ones (true + N(0,40))."""
+    scheduled; the predictions themselves are the synthetic ones (true + N(0,40)).  Two variants of the
+    generation that follows: prompts recomputed (the paper's choice, App. C), and prompts kept from the
+    perception pass as key/value pages from which every generation batch resumes."""
     shape = synth.LLAMA_7B
     kv_tok = 2 * shape.d_model * 2 * shape.n_layers
-    eng = make_engine(shape, api.runtime_cfg(256, 768, 16384, 512, int(120e9 // kv_tok)), seed=1234, device=device)
+    budget = int(55e9)                                   # batches; the kept prompts (about 90 GB) share the 150 GB pool
+    eng = make_engine(shape, api.runtime_cfg(256, 768, 16384, 512, int(150e9 // kv_tok)), seed=1234, device=device)
     g = synth.group_7b_1024(seed=0)
+    sched_cfg = api.sched_cfg(use_vbs=True, kv_budget_bytes=budget, kv_bytes_per_token=kv_tok)
     vanilla = run_group_arm(eng, api, g, api.sched_cfg(vanilla=True), synth.make_permutation(g.n, 0))
-    sched = run_group_arm(eng, api, g, api.sched_cfg(use_vbs=True, kv_budget_bytes=int(120e9), kv_bytes_per_token=kv_tok), None)
+    sched = run_group_arm(eng, api, g, sched_cfg, None)
     rng = np.random.Generator(np.random.Philox(7))
     suffix = 32
     plen = g.prompt_len + suffix
@@ -478,23 +524,37 @@ def run_perception(api, device):
         toks[off[i] + g.prompt_len[i]:off[i + 1]] = extra
     three = np.full(g.n, 3, dtype=np.int32)
     cfg = api.sched_cfg(vanilla=True, base_batch=256, max_new_tokens=4)
-    t0 = time.time()
-    res = api.ss_run_group(eng, cfg, toks, off, three, np.arange(g.n, dtype=np.int32), three)
-    wall = time.time() - t0
-    st = res["stats"]
-    perc_s = (st["prefill_ms"] + st["decode_ms"]) / 1e3
+
+    def perception_pass():
+        t0 = time.time()
+        res = api.ss_run_group(eng, cfg, toks, off, three, np.arange(g.n, dtype=np.int32), three)
+        st = res["stats"]
+        return {"device_s": (st["prefill_ms"] + st["decode_ms"]) / 1e3, "wall_s": time.time() - t0,
+                "prefill_s": st["prefill_ms"] / 1e3, "decode_s": st["decode_ms"] / 1e3, "batches": st["n_batches"],
+                "steps": st["steps"], "prompt_tokens": int(off[-1])}
+
+    perc = perception_pass()
+    # the same pass keeping every query's prompt pages, then the generation resumed from them
+    api.ss_set_prompt_cache(eng, 1, g.prompt_len)
+    perc_keep = perception_pass()
+    api.ss_set_prompt_cache(eng, 2)
+    reuse = run_group_arm(eng, api, g, sched_cfg, None)
+    api.ss_set_prompt_cache(eng, 0)
+    api.ss_drop_prompts(eng)
     useful = float(g.true_len.sum())
     return {"metric": METRIC, "unit": "tokens/s", "n_gpus": 1, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": "llama7b-shape bf16, 1024 queries; perception pass = prompt + 32 tokens, 3 generated, batches of 256"},
-            "value": useful / (perc_s + sched["device_s"]),
+            "value": useful / (perc["device_s"] + sched["device_s"]),
             "vanilla_tokens_per_s": vanilla["tokens_per_s"], "scheduled_tokens_per_s": sched["tokens_per_s"],
-            "perception": {"device_s": perc_s, "wall_s": wall, "prefill_s": st["prefill_ms"] / 1e3,
-                           "decode_s": st["decode_ms"] / 1e3, "batches": st["n_batches"], "steps": st["steps"],
-                           "prompt_tokens": int(off[-1])},
+            "perception": perc, "perception_keeping_prompts": perc_keep,
             "scheduled_device_s": sched["device_s"], "vanilla_device_s": vanilla["device_s"],
-            "overhead_of_scheduled_run": perc_s / sched["device_s"],
+            "scheduled_from_kept_prompts": {"device_s": reuse["device_s"], "prefill_s": reuse["prefill_s"],
+                                            "decode_s": reuse["decode_s"], "steps": reuse["steps"],
+                                            "kept_prompt_gb": float(np.ceil(g.prompt_len / 32).sum() * 32 * kv_tok / 1e9)},
+            "overhead_of_scheduled_run": perc["device_s"] / sched["device_s"],
             "gain_vs_vanilla_without_perception": sched["tokens_per_s"] / vanilla["tokens_per_s"],
-            "gain_vs_vanilla_with_perception": vanilla["device_s"] / (perc_s + sched["device_s"])}
+            "gain_vs_vanilla_with_perception": vanilla["device_s"] / (perc["device_s"] + sched["device_s"]),
+            "gain_vs_vanilla_with_perception_and_kept_prompts": vanilla["device_s"] / (perc_keep["device_s"] + reuse["device_s"])}
 
 
 def run_sweep(api, device, peak):
@@ -556,6 +616,8 @@ def main():
                     help="instead of the batch-16 workload: scheduled vs vanilla over the group size (7B shape)")
     ap.add_argument("--group-dispatch", action="store_true",
                     help="instead of the batch-16 workload: one 1024-query group dealt to the --gpus replicas")
+    ap.add_argument("--cpu-extras", action="store_true",
+                    help="CPU only: the oracle on configuration 1 end to end and the scheduler oracle on configurations 3-5")
     ap.add_argument("--layers", type=int, default=0, help="debug: truncate the model (invalidates the number)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
@@ -566,6 +628,10 @@ def main():
 
     if args.impl == "reference":
         run_reference(args, rank)
+        return
+    if args.cpu_extras:
+        if rank == 0:
+            print(json.dumps(run_cpu_extras()), flush=True)
         return
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         sys.exit(spawn_replicas(args.gpus))

@@ -183,6 +183,27 @@ int ss_set_sampling(ss_ctx* ctx, float temperature, uint64_t seed);
  * row's query index.  Infrastructure of the sampling above, no passage of its own. */
 int ss_set_row_keys(ss_ctx* ctx, const int32_t* keys, int32_t n);
 
+/* Prompt reuse (App. C of the paper weighs keeping the instruction's keys and values, computed once for the
+ * length-perception pass, against recomputing them for the generation; on its 80 GB GPU it recomputes.  Here the
+ * paged cache makes keeping them a matter of not returning pages.)
+ * ss_keep_prompts(): while a batch started by ss_prefill() is in flight, take over the pages that hold the first
+ *   keep_len[r] tokens of row r (2 <= keep_len[r] <= its prompt length) under the caller's id ids[r] (host int32 [B],
+ *   distinct); they stay out of the pool after ss_release_batch().  An id kept before is replaced.
+ * ss_resume(): starts a batch of B rows from kept prompts instead of a prompt pass: row r stands one token before
+ *   the end of kept prompt ids[r], feeds that token again and produces its first token with an ordinary decode step
+ *   (so a resumed batch needs cap decode steps where a prefilled one needs cap - 1).  eos_at, cap, opts,
+ *   first_tokens as for ss_prefill().  SS_ERR_STATE if an id is not kept, SS_ERR_KV_BUDGET if the pages for the rest
+ *   of the rows' contexts do not fit.  The kept pages stay kept: a row can be resumed again (recomputation).
+ * ss_drop_prompts(): returns kept pages to the pool (n = -1: all of them).  Not while a batch is in flight.
+ * ss_set_prompt_cache(): what ss_run_group() / ss_run_batches() do with the above: 0 nothing (default); 1 keep the
+ *   first keep_len[q] tokens of every query q they process (keep_len host int32 [n], copied); 2 start every batch
+ *   whose queries all have a kept prompt with ss_resume(). */
+int ss_keep_prompts(ss_ctx* ctx, const int32_t* ids, const int32_t* keep_len);
+int ss_resume(ss_ctx* ctx, const int32_t* ids, int32_t B, const int32_t* eos_at, int32_t cap, const ss_step_opts* opts,
+              int32_t* first_tokens);
+int ss_drop_prompts(ss_ctx* ctx, const int32_t* ids, int32_t n);
+int ss_set_prompt_cache(ss_ctx* ctx, int32_t mode, const int32_t* keep_len, int32_t n);
+
 /* One decode step for every active row (App. D: one token per step against the cached keys
  * and values): feed the row's last token at its next position, append its key/value, attend
  * over the row's own cache (per-row length; finished rows are skipped), project, pick the

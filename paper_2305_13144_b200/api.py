@@ -23,7 +23,8 @@ EXPORTS = [
     "ss_arena_bytes", "ss_create", "ss_destroy", "ss_load_weights", "ss_schedule", "ss_prefill",
     "ss_decode_step", "ss_decode_steps", "ss_read_batch", "ss_release_batch", "ss_run_group",
     "ss_step_model_bytes", "ss_strerror", "ss_last_device_status", "ss_last_cuda_error", "ss_kernel_launches",
-    "ss_logits_noalloc", "ss_step_trace", "ss_set_trace", "ss_set_sampling", "ss_set_row_keys", "ss_run_batches", "ss_deal_batches", "ss_set_wait_limit_ms", "ss_selftest_wait_timeout",
+    "ss_logits_noalloc", "ss_step_trace", "ss_set_trace", "ss_set_sampling", "ss_set_row_keys", "ss_run_batches", "ss_deal_batches", "ss_keep_prompts", "ss_resume", "ss_drop_prompts",
+    "ss_set_prompt_cache", "ss_set_wait_limit_ms", "ss_selftest_wait_timeout",
 ]
 
 
@@ -107,6 +108,10 @@ def lib() -> C.CDLL:
                                     [C.c_void_p] * 6 + [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
         L.ss_deal_batches.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int64, C.c_int64, C.c_int32,
                                       C.c_void_p]
+        L.ss_keep_prompts.argtypes = [C.c_void_p] * 3
+        L.ss_resume.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p]
+        L.ss_drop_prompts.argtypes = [C.c_void_p, C.c_void_p, C.c_int32]
+        L.ss_set_prompt_cache.argtypes = [C.c_void_p, C.c_int32, C.c_void_p, C.c_int32]
         L.ss_step_model_bytes.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(C.c_double)]
         L.ss_last_device_status.argtypes = [C.c_void_p, C.POINTER(C.c_uint32)]
         L.ss_step_trace.argtypes = [C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(C.c_int32)]
@@ -251,6 +256,33 @@ def ss_prefill(ctx: Ctx, tokens, cu_seqlens, eos_at, cap: int, *, forced_tokens=
     o = _opts(forced_tokens, dump_logits, dump_hidden, dump_choice)
     _check(lib().ss_prefill(ctx.handle, _hp(tk), _hp(cu), int(cu.shape[0]) - 1, _hp(ea), int(cap),
                             C.byref(o) if o else None, _dp(first_tokens)), "ss_prefill", ctx)
+
+
+def ss_keep_prompts(ctx: Ctx, ids, keep_len) -> None:
+    i, k = _np(ids, np.int32), _np(keep_len, np.int32)
+    _check(lib().ss_keep_prompts(ctx.handle, _hp(i), _hp(k)), "ss_keep_prompts", ctx)
+
+
+def ss_resume(ctx: Ctx, ids, eos_at, cap: int, *, forced_tokens=None, dump_logits=None, dump_hidden=None,
+              dump_choice=None, first_tokens=None) -> None:
+    i, ea = _np(ids, np.int32), _np(eos_at, np.int32)
+    o = _opts(forced_tokens, dump_logits, dump_hidden, dump_choice)
+    _check(lib().ss_resume(ctx.handle, _hp(i), int(i.shape[0]), _hp(ea), int(cap), C.byref(o) if o else None,
+                           _dp(first_tokens)), "ss_resume", ctx)
+
+
+def ss_drop_prompts(ctx: Ctx, ids=None) -> None:
+    if ids is None:
+        _check(lib().ss_drop_prompts(ctx.handle, None, -1), "ss_drop_prompts", ctx)
+    else:
+        i = _np(ids, np.int32)
+        _check(lib().ss_drop_prompts(ctx.handle, _hp(i), int(i.shape[0])), "ss_drop_prompts", ctx)
+
+
+def ss_set_prompt_cache(ctx: Ctx, mode: int, keep_len=None) -> None:
+    k = _np(keep_len, np.int32)
+    _check(lib().ss_set_prompt_cache(ctx.handle, int(mode), _hp(k), 0 if k is None else int(k.shape[0])),
+           "ss_set_prompt_cache", ctx)
 
 
 def ss_decode_step(ctx: Ctx, *, forced_tokens=None, dump_logits=None, dump_hidden=None, dump_choice=None,

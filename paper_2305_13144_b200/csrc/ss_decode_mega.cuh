@@ -971,6 +971,16 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
           sm->w_issued = gi + 1;
         }
       }
+      if (!ok || sm->abort) {
+        // The step was abandoned.  Before this CTA gives its shared memory up, the bulk copies it still has in
+        // flight (at most the last S ring stages) are given time to land: a bounded look at each stage's barrier,
+        // which flips once the stage's bytes are in (a stage whose activation block was never requested does not
+        // flip; its weight block has landed long before the limit, a thousand times a copy's latency, runs out).
+        for (int j = gi > S ? gi - S : 0; j < gi; ++j) {
+          const long long t0 = clock64();
+          while (!mbar_try_wait(smem_u32(&sm->full[j % S]), (uint32_t)((j / S) & 1)) && clock64() - t0 < 2000000LL) __nanosleep(100);
+        }
+      }
     }
   } else if (warp == 2) {
     // ===================== activation loader =====================

@@ -303,7 +303,7 @@ gemm_wx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
                     tok_tile * p.NT, hint_x);
       }
       // phase 2: steady state (second and later passes over the ring)
-      int stage = 0;
+      int stage = 0, issued = pre;
       uint32_t phase = 1u;
       for (int i = pre; i < n_it; ++i) {
         const long long it = it0 + i;
@@ -315,6 +315,16 @@ gemm_wx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
         else tma_load_2d(stage0 + stage * stage_bytes, &map_w, full, kblk * kTileK, tile * kTileM, hint_w);
         tma_load_2d(stage0 + stage * stage_bytes + a_bytes, &map_x, full, kblk * kTileK, tok_tile * p.NT, hint_x);
         if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+        ++issued;
+      }
+      if (issued < n_it) {
+        // a wait ran out and the kernel is leaving: the copies still in flight (at most one ring) get a bounded
+        // time to land before the CTA's shared memory is given up
+        for (int s2 = 0; s2 < p.stages; ++s2) {
+          const long long t0 = clock64();
+          while (!mbar_try_wait(smem_u32(&hdr->full[s2]), 0u) && !mbar_try_wait(smem_u32(&hdr->full[s2]), 1u) &&
+                 clock64() - t0 < 2000000LL) { }
+        }
       }
     }
   } else if (warp == 1) {
@@ -400,6 +410,17 @@ gemm_wx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 #pragma unroll
             for (int j = 0; j < 8; ++j)
               if (c + j < n_valid) out[(size_t)(tok0 + c + j) * a.ld_out + n] = __float2bfloat16_rn(v[j]);
+          }
+        }
+      } else if (a.mode == kGemmDirectF32) {
+        // plain fp32 store: the consumer (RoPE, SwiGLU) rounds once, after its own arithmetic
+        for (int c = 0; c < p.NT; c += 8) {
+          float v[8];
+          tmem_ld8(taddr + c, v);
+          if (n < p.n_out) {
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+              if (c + j < n_valid) a.out_f32[(size_t)(tok0 + c + j) * a.ld_out + n] = v[j];
           }
         }
       } else if (p.NT % 32 == 0) {

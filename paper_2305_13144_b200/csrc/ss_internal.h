@@ -39,7 +39,7 @@ enum : uint32_t {
 // CTA (split along K where a range ends inside a tile).  In kGemmPartial mode every (CTA,
 // tile) segment is written as an fp32 partial; the consumer kernel adds the segments of a tile
 // in CTA order, so the result does not depend on timing.
-enum GemmMode : int { kGemmPartial = 0, kGemmDirectBf16 = 1, kGemmDirectF32Add = 2 };
+enum GemmMode : int { kGemmPartial = 0, kGemmDirectBf16 = 1, kGemmDirectF32Add = 2, kGemmDirectF32 = 3 };
 
 struct GemmPlan {
   int n_out, K, n_tiles, kb;

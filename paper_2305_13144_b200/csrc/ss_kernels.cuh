@@ -300,12 +300,13 @@ gather_last_rmsnorm_kernel(const float* __restrict__ h, const int32_t* __restric
   }
 }
 
-// In-place RoPE on q and k of the packed [T, 3d] projection, and copy of k,v into the pages.
+// RoPE on q and k of the packed fp32 [T, 3d] projection, one rounding to bf16 afterwards: q, k, v go to the packed
+// bf16 [T, 3d] operand of the prompt-pass attention and k, v into the pages.
 // grid (T), block 256 = (256 / (Dh/2)) heads side by side x Dh/2 rotation pairs; the sine and cosine of a
 // (token, pair) are computed once and used for every head.  tok_row / tok_pos give each token's row in the
 // batch and position.
 __global__ void __launch_bounds__(256)
-rope_append_prefill_kernel(bf16* __restrict__ qkv, const int32_t* __restrict__ tok_row,
+rope_append_prefill_kernel(const float* __restrict__ qkv_f, bf16* __restrict__ qkv, const int32_t* __restrict__ tok_row,
                            const int32_t* __restrict__ tok_pos, RowState st, KvLayout kv, int layer,
                            const float* __restrict__ inv_freq, int d, uint32_t* status) {
   pdl_launch_dependents();
@@ -322,23 +323,28 @@ rope_append_prefill_kernel(bf16* __restrict__ qkv, const int32_t* __restrict__ t
     return;
   }
   for (int hd = hsub; hd < kv.H; hd += hpar) {
+    const float* qf = qkv_f + t * 3 * d + hd * Dh;
+    const float* kf = qf + d;
+    const float* vf = kf + d;
     bf16* q = qkv + t * 3 * d + hd * Dh;
     bf16* k = q + d;
-    const bf16* v = k + d;
-    const float q0 = __bfloat162float(q[i]), q1 = __bfloat162float(q[i + half]);
-    const float k0 = __bfloat162float(k[i]), k1 = __bfloat162float(k[i + half]);
+    bf16* v = k + d;
+    const float q0 = qf[i], q1 = qf[i + half], k0 = kf[i], k1 = kf[i + half];
     const bf16 kr0 = __float2bfloat16_rn(k0 * cs - k1 * sn), kr1 = __float2bfloat16_rn(k1 * cs + k0 * sn);
+    const bf16 v0 = __float2bfloat16_rn(vf[i]), v1 = __float2bfloat16_rn(vf[i + half]);
     q[i] = __float2bfloat16_rn(q0 * cs - q1 * sn);
     q[i + half] = __float2bfloat16_rn(q1 * cs + q0 * sn);
     k[i] = kr0;
     k[i + half] = kr1;
+    v[i] = v0;
+    v[i + half] = v1;
     bf16* kbase = kv.pool + (size_t)layer * kv.layer_stride + (size_t)page * kv.page_elems +
                   ((size_t)hd * kPageTokens + (pos % kPageTokens)) * Dh;
     bf16* vbase = kbase + (size_t)kv.H * kPageTokens * Dh;
     kbase[i] = kr0;
     kbase[i + half] = kr1;
-    vbase[i] = v[i];
-    vbase[i + half] = v[i + half];
+    vbase[i] = v0;
+    vbase[i + half] = v1;
   }
 }
 
@@ -501,18 +507,20 @@ attn_prefill_kernel(const bf16* __restrict__ qkv, const int32_t* __restrict__ cu
   }
 }
 
-// act[t][f] = silu(gu[t][f]) * gu[t][F+f] over T tokens, 8 features per thread (F a multiple of 8).
-// grid (T, ceil(F / 2048)), block 256.
+// act[t][f] = silu(gu[t][f]) * gu[t][F+f] over T tokens (gu fp32, act bf16: one rounding), 8 features per thread
+// (F a multiple of 8).  grid (T, ceil(F / 2048)), block 256.
 __global__ void __launch_bounds__(256)
-swiglu_kernel(const bf16* __restrict__ gu, bf16* __restrict__ act, int F) {
+swiglu_kernel(const float* __restrict__ gu, bf16* __restrict__ act, int F) {
   pdl_launch_dependents();
   pdl_wait();
   const size_t t = blockIdx.x;
   const int f0 = (blockIdx.y * blockDim.x + threadIdx.x) * 8;
   if (f0 >= F) return;
-  float gt[8], up[8];
-  unpack8(*reinterpret_cast<const uint4*>(gu + t * 2 * F + f0), gt);
-  unpack8(*reinterpret_cast<const uint4*>(gu + t * 2 * F + F + f0), up);
+  const float4* g4 = reinterpret_cast<const float4*>(gu + t * 2 * F + f0);
+  const float4* u4 = reinterpret_cast<const float4*>(gu + t * 2 * F + F + f0);
+  const float4 ga = g4[0], gb = g4[1], ua = u4[0], ub = u4[1];
+  const float gt[8] = {ga.x, ga.y, ga.z, ga.w, gb.x, gb.y, gb.z, gb.w};
+  const float up[8] = {ua.x, ua.y, ua.z, ua.w, ub.x, ub.y, ub.z, ub.w};
   __align__(16) bf16 ob[8];
 #pragma unroll
   for (int j = 0; j < 8; ++j) ob[j] = __float2bfloat16_rn(gt[j] / (1.f + __expf(-gt[j])) * up[j]);

@@ -153,7 +153,8 @@ struct ss_ctx {
   // prompt-pass activations (R rows)
   int R = 0;
   float* h = nullptr;
-  bf16 *x = nullptr, *qkv = nullptr, *attn_o = nullptr, *gu = nullptr, *act = nullptr;
+  bf16 *x = nullptr, *qkv = nullptr, *attn_o = nullptr, *act = nullptr;
+  float *qkv_f = nullptr, *gu = nullptr;   // q,k,v and gate/up as they leave their GEMMs (fp32: rounded once, after RoPE / SwiGLU)
   // decode activations (kMaxBatch rows)
   float* h_dec = nullptr;
   bf16 *x_dec = nullptr, *o_dec = nullptr, *act_dec = nullptr;
@@ -176,7 +177,19 @@ struct ss_ctx {
 
   // ---- page allocator
   std::vector<int32_t> free_pages;
-  std::vector<int32_t> batch_pages;
+  std::vector<int32_t> batch_pages;      // pages that go back to the pool when the batch in flight is released
+  // ---- kept prompts (App. C: the instruction's keys and values computed once, for the perception pass, and used
+  // again by the generation): pages that outlive the batch that filled them, by caller-chosen id
+  struct KeptPrompt {
+    std::vector<int32_t> pages;          // covering positions [0, len)
+    int32_t len;                         // tokens kept
+    int32_t last_tok;                    // token at position len - 1 (fed again when a batch resumes from here)
+  };
+  std::map<int32_t, KeptPrompt> kept;
+  std::vector<std::vector<int32_t>> row_pages;   // batch in flight: every row's pages in block-table order
+  std::vector<int32_t> batch_tokens, batch_cu;   // its prompts (host copy), empty for a resumed batch
+  int prompt_cache_mode = 0;                     // ss_run_group / ss_run_batches: 0 off, 1 keep, 2 resume
+  std::vector<int32_t> cache_keep_len;           // mode 1: tokens to keep per query
 
   // ---- batch state (host mirror)
   int B = 0;
@@ -290,7 +303,7 @@ struct ArenaPlan {
 struct Offsets {
   size_t embed, lm_head, final_norm, staging, staging_bytes, weights_end;
   std::vector<size_t> attn_norm, wqkv, wo, ffn_norm, wgu, wdown;
-  size_t inv_freq, status, rows, block_table, out_tokens, tok, h, x, qkv, attn_o, gu, act;
+  size_t inv_freq, status, rows, block_table, out_tokens, tok, h, x, qkv, qkv_f, attn_o, gu, act;
   size_t h_dec, x_dec, o_dec, act_dec, partial, kv;
   size_t tbl[5], tbl_lm_prompt, tile_val, tile_idx, rowss, grid_ctr, wptr, norm_ptr, trace;
   size_t partial_bytes;
@@ -340,8 +353,9 @@ void layout(const ss_model_cfg& m, const ss_runtime_cfg& rt, int n_sm, Offsets& 
   o.h = a.take((size_t)o.R * d * 4);
   o.x = a.take((size_t)o.R * d * 2);
   o.qkv = a.take((size_t)o.R * 3 * d * 2);
+  o.qkv_f = a.take((size_t)o.R * 3 * d * 4);
   o.attn_o = a.take((size_t)o.R * d * 2);
-  o.gu = a.take((size_t)o.R * 2 * F * 2);
+  o.gu = a.take((size_t)o.R * 2 * F * 4);
   o.act = a.take((size_t)o.R * F * 2);
   o.h_dec = a.take((size_t)kMaxBatch * d * 4);
   o.x_dec = a.take((size_t)kMaxBatch * d * 2);
@@ -512,17 +526,17 @@ int enqueue_prefill_chunk(ss_ctx* c, int s0, int s1, const int32_t* cu, int T) {
   const CUtensorMap *mx, *mo, *ma;
   int rc;
   if ((rc = xmap(c, 0, NT, &mx)) || (rc = xmap(c, 1, NT, &mo)) || (rc = xmap(c, 2, NT, &ma))) return rc;
-  const GemmPlan p_qkv = plan_gemm(3 * d, d, NT, tok_tiles, kGemmDirectBf16, c->n_sm);
+  const GemmPlan p_qkv = plan_gemm(3 * d, d, NT, tok_tiles, kGemmDirectF32, c->n_sm);
   const GemmPlan p_o = plan_gemm(d, d, NT, tok_tiles, kGemmDirectF32Add, c->n_sm);
-  const GemmPlan p_gu = plan_gemm(2 * F, d, NT, tok_tiles, kGemmDirectBf16, c->n_sm);
+  const GemmPlan p_gu = plan_gemm(2 * F, d, NT, tok_tiles, kGemmDirectF32, c->n_sm);
   const GemmPlan p_dn = plan_gemm(d, F, NT, tok_tiles, kGemmDirectF32Add, c->n_sm);
   const bf16* first_norm = m.n_layers ? c->layers[0].attn_norm : c->final_norm;
   SS_CUDA(c, launch(c, embed_rmsnorm_kernel, dim3(T), dim3(256), 0, (const int32_t*)c->d_tokens, (const int32_t*)nullptr,
                     (const bf16*)c->embed, first_norm, c->h, c->x, d, m.rms_eps, V));
   for (int l = 0; l < m.n_layers; ++l) {
     const LayerWeights& w = c->layers[l];
-    if ((rc = run_gemm(c, w.wqkv, *mx, p_qkv, kGemmDirectBf16, T, c->qkv, nullptr, 3 * d))) return rc;
-    SS_CUDA(c, launch(c, rope_append_prefill_kernel, dim3(T), dim3(256), 0, c->qkv, (const int32_t*)c->d_tok_row,
+    if ((rc = run_gemm(c, w.wqkv, *mx, p_qkv, kGemmDirectF32, T, nullptr, c->qkv_f, 3 * d))) return rc;
+    SS_CUDA(c, launch(c, rope_append_prefill_kernel, dim3(T), dim3(256), 0, (const float*)c->qkv_f, c->qkv, (const int32_t*)c->d_tok_row,
                       (const int32_t*)c->d_tok_pos, c->st, c->kv, l, (const float*)c->inv_freq, d, c->status));
     const dim3 ag(ceil_div(max_len, 64), H, nseq);
     if (Dh == 128)
@@ -531,8 +545,8 @@ int enqueue_prefill_chunk(ss_ctx* c, int s0, int s1, const int32_t* cu, int T) {
       SS_CUDA(c, launch(c, attn_prefill_kernel<64>, ag, dim3(128), 0, (const bf16*)c->qkv, (const int32_t*)c->d_cu, c->attn_o, d));
     if ((rc = run_gemm(c, w.wo, *mo, p_o, kGemmDirectF32Add, T, nullptr, c->h, d))) return rc;
     SS_CUDA(c, launch(c, rmsnorm_kernel, dim3(T), dim3(256), 0, (const float*)c->h, (const bf16*)w.ffn_norm, c->x, d, m.rms_eps));
-    if ((rc = run_gemm(c, w.wgu, *mx, p_gu, kGemmDirectBf16, T, c->gu, nullptr, 2 * F))) return rc;
-    SS_CUDA(c, launch(c, swiglu_kernel, dim3(T, ceil_div(F, 2048)), dim3(256), 0, (const bf16*)c->gu, c->act, F));
+    if ((rc = run_gemm(c, w.wgu, *mx, p_gu, kGemmDirectF32, T, nullptr, c->gu, 2 * F))) return rc;
+    SS_CUDA(c, launch(c, swiglu_kernel, dim3(T, ceil_div(F, 2048)), dim3(256), 0, (const float*)c->gu, c->act, F));
     if ((rc = run_gemm(c, w.wdown, *ma, p_dn, kGemmDirectF32Add, T, nullptr, c->h, d))) return rc;
     if (l + 1 < m.n_layers)
       SS_CUDA(c, launch(c, rmsnorm_kernel, dim3(T), dim3(256), 0, (const float*)c->h,
@@ -648,7 +662,8 @@ int ss_create(const ss_model_cfg* model, const ss_runtime_cfg* rt, void* dev_are
   c->x = (bf16*)(A + o.x);
   c->qkv = (bf16*)(A + o.qkv);
   c->attn_o = (bf16*)(A + o.attn_o);
-  c->gu = (bf16*)(A + o.gu);
+  c->gu = (float*)(A + o.gu);
+  c->qkv_f = (float*)(A + o.qkv_f);
   c->act = (bf16*)(A + o.act);
   c->h_dec = (float*)(A + o.h_dec);
   c->x_dec = (bf16*)(A + o.x_dec);
@@ -775,6 +790,7 @@ int ss_release_batch(ss_ctx* c) {
   if (!c) return SS_ERR_ARG;
   for (int32_t p : c->batch_pages) c->free_pages.push_back(p);
   c->batch_pages.clear();
+  c->row_pages.clear();
   c->in_batch = false;
   c->B = 0;
   return SS_OK;
@@ -805,6 +821,9 @@ int ss_prefill(ss_ctx* c, const int32_t* tokens, const int32_t* cu, int32_t B, c
   std::vector<int32_t> bt((size_t)B * c->st.max_pages, -1);
   c->batch_pages.clear();
   c->prompt_len.assign(B, 0);
+  c->row_pages.assign(B, {});
+  c->batch_tokens.assign(tokens, tokens + Ttot);
+  c->batch_cu.assign(cu, cu + B + 1);
   for (int r = 0; r < B; ++r) {
     const int len = cu[r + 1] - cu[r];
     c->prompt_len[r] = len;
@@ -813,6 +832,7 @@ int ss_prefill(ss_ctx* c, const int32_t* tokens, const int32_t* cu, int32_t B, c
       const int32_t pg = c->free_pages.back();
       c->free_pages.pop_back();
       c->batch_pages.push_back(pg);
+      c->row_pages[r].push_back(pg);
       bt[(size_t)r * c->st.max_pages + p] = pg;
     }
   }
@@ -881,6 +901,121 @@ int ss_prefill(ss_ctx* c, const int32_t* tokens, const int32_t* cu, int32_t B, c
                    (const int32_t*)c->tile_idx, c->n_tiles_lm, opts ? opts->forced_tokens : (const int32_t*)nullptr,
                    first_tokens, opts ? opts->dump_choice : (int32_t*)nullptr, B, m.eos_id, 1));
 #undef SS_CUDA_B
+  return SS_OK;
+}
+
+int ss_keep_prompts(ss_ctx* c, const int32_t* ids, const int32_t* keep_len) {
+  if (!c || !ids || !keep_len) return SS_ERR_ARG;
+  if (!c->in_batch || c->batch_cu.empty()) return SS_ERR_STATE;      // no batch, or one that was itself resumed
+  const int B = c->B;
+  for (int r = 0; r < B; ++r) {
+    if (keep_len[r] < 2 || keep_len[r] > c->prompt_len[r]) return SS_ERR_ARG;
+    for (int q = 0; q < r; ++q)
+      if (ids[q] == ids[r]) return SS_ERR_ARG;
+  }
+  for (int r = 0; r < B; ++r) {
+    auto old = c->kept.find(ids[r]);
+    if (old != c->kept.end()) {
+      for (int32_t p : old->second.pages) c->free_pages.push_back(p);
+      c->kept.erase(old);
+    }
+    const int n_keep = ceil_div(keep_len[r], kPageTokens);
+    ss_ctx::KeptPrompt k;
+    k.pages.assign(c->row_pages[r].begin(), c->row_pages[r].begin() + n_keep);
+    k.len = keep_len[r];
+    k.last_tok = c->batch_tokens[c->batch_cu[r] + keep_len[r] - 1];
+    // these pages no longer go back to the pool with the batch
+    for (int32_t p : k.pages) {
+      auto it = std::find(c->batch_pages.begin(), c->batch_pages.end(), p);
+      if (it != c->batch_pages.end()) { *it = c->batch_pages.back(); c->batch_pages.pop_back(); }
+    }
+    c->kept.emplace(ids[r], std::move(k));
+  }
+  return SS_OK;
+}
+
+int ss_drop_prompts(ss_ctx* c, const int32_t* ids, int32_t n) {
+  if (!c || n < -1 || (n > 0 && !ids)) return SS_ERR_ARG;
+  if (c->in_batch) return SS_ERR_STATE;
+  if (n == -1) {
+    for (auto& kv : c->kept)
+      for (int32_t p : kv.second.pages) c->free_pages.push_back(p);
+    c->kept.clear();
+    return SS_OK;
+  }
+  for (int i = 0; i < n; ++i) {
+    auto it = c->kept.find(ids[i]);
+    if (it == c->kept.end()) continue;
+    for (int32_t p : it->second.pages) c->free_pages.push_back(p);
+    c->kept.erase(it);
+  }
+  return SS_OK;
+}
+
+int ss_resume(ss_ctx* c, const int32_t* ids, int32_t B, const int32_t* eos_at, int32_t cap, const ss_step_opts* opts,
+              int32_t* first_tokens) {
+  if (!c || !ids || B < 1 || cap < 1) return SS_ERR_ARG;
+  if (c->n_loaded != c->n_expected || c->in_batch) return SS_ERR_STATE;
+  if (B > c->rt.max_batch || cap > c->rt.max_new_tokens) return SS_ERR_CAPACITY;
+  size_t need_pages = 0;
+  for (int r = 0; r < B; ++r) {
+    auto it = c->kept.find(ids[r]);
+    if (it == c->kept.end()) return SS_ERR_STATE;
+    for (int q = 0; q < r; ++q)
+      if (ids[q] == ids[r]) return SS_ERR_ARG;
+    const int len = it->second.len;
+    if (len + cap > c->rt.max_ctx) return SS_ERR_CAPACITY;
+    if (eos_at && eos_at[r] < 1) return SS_ERR_ARG;
+    need_pages += (size_t)ceil_div(len + cap, kPageTokens) - it->second.pages.size();
+  }
+  if (need_pages > c->free_pages.size()) return SS_ERR_KV_BUDGET;
+  std::vector<int32_t> bt((size_t)B * c->st.max_pages, -1);
+  std::vector<int32_t> rows((size_t)kMaxBatch * 8, 0);
+  c->batch_pages.clear();
+  c->batch_tokens.clear();
+  c->batch_cu.clear();
+  c->prompt_len.assign(B, 0);
+  c->row_pages.assign(B, {});
+  for (int r = 0; r < B; ++r) {
+    const ss_ctx::KeptPrompt& k = c->kept[ids[r]];
+    c->prompt_len[r] = k.len;
+    c->row_pages[r] = k.pages;
+    const int np = ceil_div(k.len + cap, kPageTokens);
+    for (int p = (int)k.pages.size(); p < np; ++p) {
+      const int32_t pg = c->free_pages.back();
+      c->free_pages.pop_back();
+      c->batch_pages.push_back(pg);
+      c->row_pages[r].push_back(pg);
+    }
+    for (int p = 0; p < np; ++p) bt[(size_t)r * c->st.max_pages + p] = c->row_pages[r][p];
+    // the row stands one token before the end of its kept prompt: that token is fed again by the first step
+    rows[0 * kMaxBatch + r] = k.len - 1;
+    rows[1 * kMaxBatch + r] = k.last_tok;
+    rows[3 * kMaxBatch + r] = 1;
+    rows[5 * kMaxBatch + r] = eos_at ? eos_at[r] : 0;
+    rows[6 * kMaxBatch + r] = r < (int)c->next_row_keys.size() ? c->next_row_keys[r] : r;
+  }
+  c->next_row_keys.clear();
+  rows[7 * kMaxBatch + 0] = cap;
+  rows[7 * kMaxBatch + 1] = B;
+  c->in_batch = true;
+  c->B = B;
+  c->cap = cap;
+  auto bail = [&](int code) { ss_release_batch(c); return code; };
+  cudaError_t e = cudaMemcpyAsync(c->st.ctx_len, rows.data(), rows.size() * 4, cudaMemcpyHostToDevice, c->stream);
+  if (e == cudaSuccess) e = cudaMemcpyAsync(c->st.block_table, bt.data(), bt.size() * 4, cudaMemcpyHostToDevice, c->stream);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(c->stream);          // the host vectors go out of scope
+  if (e != cudaSuccess) { c->last_cuda = (int)e; return bail(SS_ERR_CUDA); }
+  int rc = enqueue_decode_step(c, opts, first_tokens);
+  if (rc) return bail(rc);
+  return SS_OK;
+}
+
+int ss_set_prompt_cache(ss_ctx* c, int32_t mode, const int32_t* keep_len, int32_t n) {
+  if (!c || mode < 0 || mode > 2 || n < 0 || (mode == 1 && (!keep_len || n < 1))) return SS_ERR_ARG;
+  c->prompt_cache_mode = mode;
+  c->cache_keep_len.clear();
+  if (mode == 1) c->cache_keep_len.assign(keep_len, keep_len + n);
   return SS_OK;
 }
 
@@ -1053,9 +1188,22 @@ static int run_batch_list(ss_ctx* c, const ss_sched_cfg* cfg, const int32_t* pro
       if (eos_at) { eos_b.push_back(eos_at[q]); max_target = std::max(max_target, eos_at[q]); }
     }
     c->next_row_keys.assign(rows_src, rows_src + B);      // a row's sampling key is its query id, in every pass
+    // prompt reuse (App. C): a batch whose queries all have kept prompts starts from them instead of a prompt pass
+    bool resume = c->prompt_cache_mode == 2;
+    for (int r = 0; r < B && resume; ++r) resume = c->kept.count(rows_src[r]) != 0;
     SS_CUDA_G(cudaEventRecord(ev[0], c->stream));
-    rc = ss_prefill(c, toks.data(), cu.data(), B, eos_at ? eos_b.data() : nullptr, b.cap, nullptr, nullptr);
+    if (resume) rc = ss_resume(c, rows_src, B, eos_at ? eos_b.data() : nullptr, b.cap, nullptr, nullptr);
+    else rc = ss_prefill(c, toks.data(), cu.data(), B, eos_at ? eos_b.data() : nullptr, b.cap, nullptr, nullptr);
     if (rc) return cleanup(rc);
+    if (c->prompt_cache_mode == 1 && !resume) {
+      std::vector<int32_t> kl(B);
+      for (int r = 0; r < B; ++r) {
+        const int q = rows_src[r];
+        if (q >= (int)c->cache_keep_len.size()) return cleanup(SS_ERR_ARG);
+        kl[r] = c->cache_keep_len[q];
+      }
+      if ((rc = ss_keep_prompts(c, rows_src, kl.data()))) return cleanup(rc);
+    }
     SS_CUDA_G(cudaEventRecord(ev[1], c->stream));
     if (eos_at) {
       // lengths are forced, so the number of steps is known: the longest target or the cap
