@@ -162,6 +162,57 @@ __device__ __forceinline__ void tmem_ld64(uint32_t taddr, uint32_t (&r)[64]) {
       : "memory");
 }
 
+// ---- forms for a pair of CTAs on neighbouring SMs working on one accumulator tile (cta_group::2) ---------------
+// TMA tile load whose bytes are counted on the mbarrier of the pair's first CTA (the one that issues the MMAs):
+// both CTAs execute it with the address of their own copy of the barrier; clearing the CTA-rank bit of the
+// shared-window address makes it the first CTA's.  Every CTA loads only its own operand halves.
+constexpr uint32_t kPairLeaderMask = 0xFEFFFFFFu;
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y,
+                                                 uint64_t hint) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+      " [%0], [%1, {%3, %4}], [%2], %5;"
+      :
+      : "r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar & kPairLeaderMask), "r"(x), "r"(y), "l"(hint)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t dst_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish_pair() {
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t taddr, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+// D[tmem of both CTAs] (+)= A * B with M = 256 (128 rows from each CTA's shared memory), N from the descriptor
+// (half of the B rows from each CTA), K = 16.  Issued by one thread of the pair's first CTA.
+__device__ __forceinline__ void umma_bf16_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                               uint32_t accumulate) {
+  const uint32_t z = 0;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n\t}"
+      :
+      : "r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(z)
+      : "memory");
+}
+// Arrives on the same-named mbarrier of both CTAs of the pair once every MMA issued so far has completed.
+__device__ __forceinline__ void umma_commit_pair(uint32_t bar) {
+  const uint16_t mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"(mask) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t cluster_cta_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+
 // Shared-memory matrix descriptor: K-major tile, 128-byte swizzle, rows of 128 bytes,
 // 8-row groups 1024 bytes apart.
 __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
@@ -461,6 +512,169 @@ gemm_wx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, (uint32_t)p.tmem_cols);
+  }
+}
+
+// ------------------------------------------------------------------------------------ the paired kernel
+// The prompt-pass GEMM on pairs of CTAs (a cluster of two neighbouring SMs, tcgen05 cta_group::2): the pair
+// computes a 256-row x 256-token tile, CTA r of the pair holding weight rows 128 r .. 128 r + 127 (its half of a
+// 32 KiB block of the tiled layout) and tokens 128 r .. 128 r + 127 of the token tile in its shared memory, and
+// rows 128 r .. of the accumulator in its tensor memory.  One thread of the first CTA issues the MMAs for both.
+// Why: with one CTA per tile, 48 KiB written into shared memory and 48 KiB read out of it by the tensor core per
+// k-block exceed what the shared memory of one SM moves in the 512 cycles the four MMAs take; in the pair every
+// CTA stages 32 KiB per k-block for the same arithmetic.
+// grid (2 * token tiles of 256, ceil(n_out / 256)), cluster (2, 1, 1); one accumulator tile per CTA.
+constexpr int kPairStageBytes = 2 * kTileM * kTileK * 2;        // 16 KiB of weights + 16 KiB of activations
+constexpr int kPairTokens = 256;                                 // token tile of the pair (128 per CTA)
+
+static __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
+gemm_wx_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, GemmArgs a) {
+  extern __shared__ uint8_t smem_raw[];
+  const GemmPlan& p = a.p;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_cta_rank();          // 0: issues the MMAs; 1: its partner
+  // blockIdx.x = 2 * token tile + rank, blockIdx.y = pair of weight tiles: CTAs that follow each other in launch
+  // order read the same weight block, so it crosses HBM once and is served from L2 to the other token tiles
+  const int tile = 2 * (int)blockIdx.y + (int)rank;  // 128-row weight tile of this CTA (pair = tiles 2j, 2j + 1)
+  const int tok_tile = blockIdx.x >> 1;
+  GemmSmemHeader* hdr = reinterpret_cast<GemmSmemHeader*>(smem_raw);
+  const uint32_t stage0 = (smem_u32(smem_raw) + (uint32_t)sizeof(GemmSmemHeader) + 1023u) & ~1023u;
+  const uint32_t a_bytes = kTileM * kTileK * 2;
+  const int n_it = p.kb;
+
+  if (threadIdx.x == 0) {
+    pdl_launch_dependents();
+    for (int s = 0; s < p.stages; ++s) {
+      mbar_init(smem_u32(&hdr->full[s]), 1);
+      mbar_init(smem_u32(&hdr->empty[s]), 1);
+    }
+    mbar_init(smem_u32(&hdr->acc_full[0]), 1);
+    fence_barrier_init();
+    tma_prefetch_desc(&map_w);
+    tma_prefetch_desc(&map_x);
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(smem_u32(&hdr->tmem_base), (uint32_t)kPairTokens);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();                                // both CTAs' barriers exist before either signals the other's
+  tc_fence_after();
+  const uint32_t tmem_base = hdr->tmem_base;
+
+  if (warp == 0) {
+    // ===================== TMA producer (one per CTA) =====================
+    if (lane == 0) {
+      uint64_t hint_w, hint_x;
+      asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(hint_w));
+      asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(hint_x));
+      // the tiled weights seen as lines of 128 bytes: this CTA's half of block (tile / 2, k) starts at line
+      // ((tile / 2) * kb + k) * 256 + (tile & 1) * 128 and is 128 lines long
+      const int line0 = (tile >> 1) * p.kb * kTileN + (tile & 1) * kTileM;
+      const int tok0 = tok_tile * kPairTokens + (int)rank * (kPairTokens / 2);
+      pdl_wait();
+      int stage = 0;
+      uint32_t phase = 0;
+      int issued = 0;
+      for (int i = 0; i < n_it; ++i) {
+        if (i >= p.stages && !mbar_wait(smem_u32(&hdr->empty[stage]), phase ^ 1u, a.status, kStatusProducerTimeout)) break;
+        const uint32_t full = smem_u32(&hdr->full[stage]);
+        // the first CTA's barrier counts the bytes of all four loads of the stage (two per CTA)
+        if (rank == 0) mbar_expect_tx(full, 2u * kPairStageBytes);
+        const uint32_t dst = stage0 + (uint32_t)stage * kPairStageBytes;
+        tma_load_2d_pair(dst, &map_w, full, 0, line0 + i * kTileN, hint_w);
+        tma_load_2d_pair(dst + a_bytes, &map_x, full, i * kTileK, tok0, hint_x);
+        ++issued;
+        if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+      }
+      if (issued < n_it) {
+        // a wait ran out: give the copies in flight a bounded time to land before the shared memory is given up
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) { }
+      }
+    }
+  } else if (warp == 1) {
+    // ===================== MMA issuer (first CTA of the pair only) =====================
+    if (lane == 0 && rank == 0) {
+      const uint32_t idesc = umma_idesc_bf16(kPairTokens, 256);
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int i = 0; i < n_it; ++i) {
+        ok = mbar_wait(smem_u32(&hdr->full[stage]), phase, a.status, kStatusMmaTimeout);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t sa = stage0 + (uint32_t)stage * kPairStageBytes;
+        const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sa + a_bytes);
+#pragma unroll
+        for (int k = 0; k < kTileK / 16; ++k)
+          umma_bf16_pair(tmem_base, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (i == 0 && k == 0) ? 0u : 1u);
+        umma_commit_pair(smem_u32(&hdr->empty[stage]));      // frees the stage in both CTAs when these MMAs retire
+        if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+      }
+      if (ok) umma_commit_pair(smem_u32(&hdr->acc_full[0]));
+    }
+  } else {
+    // ===================== epilogue (4 warps, one TMEM lane quarter each): this CTA's 128 rows x 256 tokens ====
+    pdl_wait();
+    const int quarter = warp & 3;
+    const int row = quarter * 32 + lane;
+    const int tok0 = tok_tile * kPairTokens;
+    int n_valid = a.n_tok - tok0;
+    if (n_valid > kPairTokens) n_valid = kPairTokens;
+    bool ok = mbar_wait(smem_u32(&hdr->acc_full[0]), 0u, a.status, kStatusEpilogueTimeout);
+    ok = __all_sync(0xffffffffu, ok);
+    if (ok) {
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+      const int n = tile * kTileM + row;
+      if (a.mode == kGemmDirectF32) {
+        for (int c = 0; c < kPairTokens; c += 32) {
+          float v[32];
+          tmem_ld32(taddr + c, v);
+          if (n < p.n_out) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (c + j < n_valid) a.out_f32[(size_t)(tok0 + c + j) * a.ld_out + n] = v[j];
+          }
+        }
+      } else if (a.mode == kGemmDirectBf16) {
+        __nv_bfloat16* out = reinterpret_cast<__nv_bfloat16*>(a.out_bf16);
+        for (int c = 0; c < kPairTokens; c += 32) {
+          float v[32];
+          tmem_ld32(taddr + c, v);
+          if (n < p.n_out) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (c + j < n_valid) out[(size_t)(tok0 + c + j) * a.ld_out + n] = __float2bfloat16_rn(v[j]);
+          }
+        }
+      } else {
+        // read-modify-write of the fp32 residual: 32 tokens' loads in flight per round trip
+        for (int c = 0; c < kPairTokens; c += 32) {
+          float v[32], h[32];
+          tmem_ld32(taddr + c, v);
+          if (n < p.n_out) {
+            float* o = a.out_f32 + (size_t)(tok0 + c) * a.ld_out + n;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) h[j] = (c + j < n_valid) ? __ldcg(o + (size_t)j * a.ld_out) : 0.f;
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (c + j < n_valid) o[(size_t)j * a.ld_out] = h[j] + v[j];
+          }
+        }
+      }
+    }
+  }
+
+  // neither CTA may give up its shared or tensor memory while the other's MMAs or copies can still touch it
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc_pair(tmem_base, (uint32_t)kPairTokens);
   }
 }
 

@@ -174,6 +174,8 @@ struct ss_ctx {
   int n_tiles_lm = 0;
   // tensor maps for activation operands, keyed by (buffer id, box rows)
   std::map<std::pair<int, int>, CUtensorMap> xmaps;
+  // the tiled projection matrices seen as lines of 128 bytes (for the paired prompt-pass GEMM), [4 * layer + type]
+  std::vector<CUtensorMap> wmaps;
 
   // ---- page allocator
   std::vector<int32_t> free_pages;
@@ -245,6 +247,23 @@ int make_map(ss_ctx* c, CUtensorMap* out, const void* base, int64_t rows, int64_
   return SS_OK;
 }
 
+// A tiled weight matrix as a 2-D tensor of 128-byte lines (64 bf16 each); box = 128 lines = one CTA's half of a block.
+// The lines already hold the swizzled shared-memory image, so the copy itself does not swizzle.
+int make_line_map(ss_ctx* c, CUtensorMap* out, const void* base, size_t bytes) {
+  cuuint64_t dims[2] = {(cuuint64_t)kTileK, (cuuint64_t)(bytes / 128)};
+  cuuint64_t strides[1] = {128};
+  cuuint32_t box[2] = {(cuuint32_t)kTileK, (cuuint32_t)kTileM};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = c->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    c->last_cuda = (int)r;
+    return SS_ERR_CUDA;
+  }
+  return SS_OK;
+}
+
 // activation operand map (cached): id 0 = x, 1 = attn_o, 2 = act (prompt pass); 3 = x_dec, 4 = o_dec, 5 = act_dec
 int xmap(ss_ctx* c, int id, int box_rows, const CUtensorMap** out) {
   auto key = std::make_pair(id, box_rows);
@@ -288,6 +307,28 @@ int run_gemm(ss_ctx* c, const uint8_t* w_tiled, const CUtensorMap& mx, const Gem
   }
   // the weight tensor map is unused with tiled weights; the activation map stands in for it
   SS_CUDA(c, launch(c, gemm_wx_kernel, dim3(p.gridy, p.gridx), dim3(kGemmThreads), (size_t)p.smem_bytes, mx, mx, a));
+  return SS_OK;
+}
+
+// The same product on pairs of CTAs (gemm_wx_pair_kernel): token tiles of 256, direct epilogues only.
+int run_gemm_pair(ss_ctx* c, const CUtensorMap& mw, const CUtensorMap& mx, int n_out, int K, int mode, int n_tok,
+                  void* out_bf16, float* out_f32, int ld_out) {
+  GemmArgs a{};
+  a.p.n_out = n_out;
+  a.p.K = K;
+  a.p.n_tiles = 2 * ceil_div(n_out, kTileN);
+  a.p.kb = ceil_div(K, kTileK);
+  a.p.NT = kPairTokens;
+  a.p.stages = std::min(kGemmMaxStages, (227 * 1024 - 2048) / kPairStageBytes);
+  a.p.smem_bytes = 2048 + a.p.stages * kPairStageBytes;
+  a.mode = mode;
+  a.n_tok = n_tok;
+  a.out_bf16 = out_bf16;
+  a.out_f32 = out_f32;
+  a.ld_out = ld_out;
+  a.status = c->status;
+  SS_CUDA(c, launch(c, gemm_wx_pair_kernel, dim3(2 * ceil_div(n_tok, kPairTokens), a.p.n_tiles / 2), dim3(kGemmThreads),
+                    (size_t)a.p.smem_bytes, mw, mx, a));
   return SS_OK;
 }
 
@@ -521,7 +562,9 @@ int enqueue_prefill_chunk(ss_ctx* c, int s0, int s1, const int32_t* cu, int T) {
   const int nseq = s1 - s0;
   int max_len = 0;
   for (int s = s0; s < s1; ++s) max_len = std::max(max_len, cu[s + 1] - cu[s]);
-  const int NT = std::min(256, round_up(T, 16));
+  // more than half a pair's token tile: the paired kernel (token tiles of 256, two CTAs per 256 x 256 tile)
+  const bool pair = T > kPairTokens / 2;
+  const int NT = pair ? kPairTokens / 2 : std::min(256, round_up(T, 16));
   const int tok_tiles = ceil_div(T, NT);
   const CUtensorMap *mx, *mo, *ma;
   int rc;
@@ -530,12 +573,18 @@ int enqueue_prefill_chunk(ss_ctx* c, int s0, int s1, const int32_t* cu, int T) {
   const GemmPlan p_o = plan_gemm(d, d, NT, tok_tiles, kGemmDirectF32Add, c->n_sm);
   const GemmPlan p_gu = plan_gemm(2 * F, d, NT, tok_tiles, kGemmDirectF32, c->n_sm);
   const GemmPlan p_dn = plan_gemm(d, F, NT, tok_tiles, kGemmDirectF32Add, c->n_sm);
+  // one projection: on pairs of CTAs, or one CTA per tile for short chunks
+  auto project = [&](int l, int type, const uint8_t* w, const CUtensorMap& act, const GemmPlan& pl, int n_out, int K,
+                     int mode, float* out, int ld) -> int {
+    if (pair) return run_gemm_pair(c, c->wmaps[4 * l + type], act, n_out, K, mode, T, nullptr, out, ld);
+    return run_gemm(c, w, act, pl, mode, T, nullptr, out, ld);
+  };
   const bf16* first_norm = m.n_layers ? c->layers[0].attn_norm : c->final_norm;
   SS_CUDA(c, launch(c, embed_rmsnorm_kernel, dim3(T), dim3(256), 0, (const int32_t*)c->d_tokens, (const int32_t*)nullptr,
                     (const bf16*)c->embed, first_norm, c->h, c->x, d, m.rms_eps, V));
   for (int l = 0; l < m.n_layers; ++l) {
     const LayerWeights& w = c->layers[l];
-    if ((rc = run_gemm(c, w.wqkv, *mx, p_qkv, kGemmDirectF32, T, nullptr, c->qkv_f, 3 * d))) return rc;
+    if ((rc = project(l, 0, w.wqkv, *mx, p_qkv, 3 * d, d, kGemmDirectF32, c->qkv_f, 3 * d))) return rc;
     SS_CUDA(c, launch(c, rope_append_prefill_kernel, dim3(T), dim3(256), 0, (const float*)c->qkv_f, c->qkv, (const int32_t*)c->d_tok_row,
                       (const int32_t*)c->d_tok_pos, c->st, c->kv, l, (const float*)c->inv_freq, d, c->status));
     const dim3 ag(ceil_div(max_len, 64), H, nseq);
@@ -543,11 +592,11 @@ int enqueue_prefill_chunk(ss_ctx* c, int s0, int s1, const int32_t* cu, int T) {
       SS_CUDA(c, launch(c, attn_prefill_kernel<128>, ag, dim3(128), 0, (const bf16*)c->qkv, (const int32_t*)c->d_cu, c->attn_o, d));
     else
       SS_CUDA(c, launch(c, attn_prefill_kernel<64>, ag, dim3(128), 0, (const bf16*)c->qkv, (const int32_t*)c->d_cu, c->attn_o, d));
-    if ((rc = run_gemm(c, w.wo, *mo, p_o, kGemmDirectF32Add, T, nullptr, c->h, d))) return rc;
+    if ((rc = project(l, 1, w.wo, *mo, p_o, d, d, kGemmDirectF32Add, c->h, d))) return rc;
     SS_CUDA(c, launch(c, rmsnorm_kernel, dim3(T), dim3(256), 0, (const float*)c->h, (const bf16*)w.ffn_norm, c->x, d, m.rms_eps));
-    if ((rc = run_gemm(c, w.wgu, *mx, p_gu, kGemmDirectF32, T, nullptr, c->gu, 2 * F))) return rc;
+    if ((rc = project(l, 2, w.wgu, *mx, p_gu, 2 * F, d, kGemmDirectF32, c->gu, 2 * F))) return rc;
     SS_CUDA(c, launch(c, swiglu_kernel, dim3(T, ceil_div(F, 2048)), dim3(256), 0, (const float*)c->gu, c->act, F));
-    if ((rc = run_gemm(c, w.wdown, *ma, p_dn, kGemmDirectF32Add, T, nullptr, c->h, d))) return rc;
+    if ((rc = project(l, 3, w.wdown, *ma, p_dn, d, F, kGemmDirectF32Add, c->h, d))) return rc;
     if (l + 1 < m.n_layers)
       SS_CUDA(c, launch(c, rmsnorm_kernel, dim3(T), dim3(256), 0, (const float*)c->h,
                         (const bf16*)c->layers[l + 1].attn_norm, c->x, d, m.rms_eps));
@@ -692,6 +741,14 @@ int ss_create(const ss_model_cfg* model, const ss_runtime_cfg* rt, void* dev_are
         cudaMemset(A + o.rowss, 0, o.wptr - o.rowss) != cudaSuccess)
       return fail(SS_ERR_CUDA);
   }
+  c->wmaps.resize((size_t)4 * model->n_layers);
+  for (int l = 0; l < model->n_layers; ++l) {
+    const LayerWeights& w = c->layers[l];
+    const uint8_t* base[4] = {w.wqkv, w.wo, w.wgu, w.wdown};
+    const size_t bytes[4] = {tiled_bytes(3 * d, d), tiled_bytes(d, d), tiled_bytes(2 * F, d), tiled_bytes(d, F)};
+    for (int t = 0; t < 4; ++t)
+      if (int rc2 = make_line_map(c, &c->wmaps[4 * l + t], base[t], bytes[t])) return fail(rc2);
+  }
   c->tile_val = (float*)(A + o.tile_val);
   c->tile_idx = (int32_t*)(A + o.tile_idx);
   c->n_tiles_lm = ceil_div((int)V, kTileM);
@@ -730,6 +787,8 @@ int ss_create(const ss_model_cfg* model, const ss_runtime_cfg* rt, void* dev_are
   if (e == cudaSuccess) e = cudaHostAlloc((void**)&c->pinned, 64, cudaHostAllocDefault);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(gemm_wx_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(gemm_wx_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(decode_step_mega_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e == cudaSuccess)
