@@ -523,24 +523,30 @@ gemm_wx_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 // Why: with one CTA per tile, 48 KiB written into shared memory and 48 KiB read out of it by the tensor core per
 // k-block exceed what the shared memory of one SM moves in the 512 cycles the four MMAs take; in the pair every
 // CTA stages 32 KiB per k-block for the same arithmetic.
-// grid (2 * token tiles of 256, ceil(n_out / 256)), cluster (2, 1, 1); one accumulator tile per CTA.
 constexpr int kPairStageBytes = 2 * kTileM * kTileK * 2;        // 16 KiB of weights + 16 KiB of activations
 constexpr int kPairTokens = 256;                                 // token tile of the pair (128 per CTA)
 
+// Remote arrival on the first CTA's copy of a barrier (used by the partner's epilogue warps).
+__device__ __forceinline__ void mbar_arrive_leader(uint32_t bar) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar & kPairLeaderMask) : "memory");
+}
+
+// Persistent: gridDim.x / 2 pairs walk the (pair of weight tiles, token tile) units pair, pair + P, pair + 2 P, ...
+// with the token tile as the fast index (pairs that run side by side read the same weight block: it crosses HBM
+// once).  Two accumulator buffers of 256 columns: the drain of one unit overlaps the MMAs of the next.
 static __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kGemmThreads, 1)
 gemm_wx_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, GemmArgs a) {
   extern __shared__ uint8_t smem_raw[];
   const GemmPlan& p = a.p;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t rank = cluster_cta_rank();          // 0: issues the MMAs; 1: its partner
-  // blockIdx.x = 2 * token tile + rank, blockIdx.y = pair of weight tiles: CTAs that follow each other in launch
-  // order read the same weight block, so it crosses HBM once and is served from L2 to the other token tiles
-  const int tile = 2 * (int)blockIdx.y + (int)rank;  // 128-row weight tile of this CTA (pair = tiles 2j, 2j + 1)
-  const int tok_tile = blockIdx.x >> 1;
+  const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+  const int tok_tiles = p.gridy;                     // token tiles of 256
+  const int n_units = (p.n_tiles >> 1) * tok_tiles;
   GemmSmemHeader* hdr = reinterpret_cast<GemmSmemHeader*>(smem_raw);
   const uint32_t stage0 = (smem_u32(smem_raw) + (uint32_t)sizeof(GemmSmemHeader) + 1023u) & ~1023u;
   const uint32_t a_bytes = kTileM * kTileK * 2;
-  const int n_it = p.kb;
+  const int kb = p.kb;
 
   if (threadIdx.x == 0) {
     pdl_launch_dependents();
@@ -548,13 +554,16 @@ gemm_wx_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
       mbar_init(smem_u32(&hdr->full[s]), 1);
       mbar_init(smem_u32(&hdr->empty[s]), 1);
     }
-    mbar_init(smem_u32(&hdr->acc_full[0]), 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(smem_u32(&hdr->acc_full[b]), 1);
+      mbar_init(smem_u32(&hdr->acc_empty[b]), 8);    // four epilogue warps of each CTA (used in the first CTA only)
+    }
     fence_barrier_init();
     tma_prefetch_desc(&map_w);
     tma_prefetch_desc(&map_x);
   }
   if (warp == 1) {
-    tmem_alloc_pair(smem_u32(&hdr->tmem_base), (uint32_t)kPairTokens);
+    tmem_alloc_pair(smem_u32(&hdr->tmem_base), 2u * kPairTokens);
     tmem_relinquish_pair();
   }
   tc_fence_before();
@@ -569,26 +578,28 @@ gemm_wx_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
       uint64_t hint_w, hint_x;
       asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(hint_w));
       asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(hint_x));
-      // the tiled weights seen as lines of 128 bytes: this CTA's half of block (tile / 2, k) starts at line
-      // ((tile / 2) * kb + k) * 256 + (tile & 1) * 128 and is 128 lines long
-      const int line0 = (tile >> 1) * p.kb * kTileN + (tile & 1) * kTileM;
-      const int tok0 = tok_tile * kPairTokens + (int)rank * (kPairTokens / 2);
       pdl_wait();
-      int stage = 0;
+      int stage = 0, gi = 0;
       uint32_t phase = 0;
-      int issued = 0;
-      for (int i = 0; i < n_it; ++i) {
-        if (i >= p.stages && !mbar_wait(smem_u32(&hdr->empty[stage]), phase ^ 1u, a.status, kStatusProducerTimeout)) break;
-        const uint32_t full = smem_u32(&hdr->full[stage]);
-        // the first CTA's barrier counts the bytes of all four loads of the stage (two per CTA)
-        if (rank == 0) mbar_expect_tx(full, 2u * kPairStageBytes);
-        const uint32_t dst = stage0 + (uint32_t)stage * kPairStageBytes;
-        tma_load_2d_pair(dst, &map_w, full, 0, line0 + i * kTileN, hint_w);
-        tma_load_2d_pair(dst + a_bytes, &map_x, full, i * kTileK, tok0, hint_x);
-        ++issued;
-        if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+      bool ok = true;
+      for (int u = pair; u < n_units && ok; u += n_pairs) {
+        const int wt = u / tok_tiles, tt = u - wt * tok_tiles;
+        // the tiled weights seen as lines of 128 bytes: this CTA's half of block (wt, k) starts at line
+        // (wt * kb + k) * 256 + rank * 128 and is 128 lines long
+        const int line0 = wt * kb * kTileN + (int)rank * kTileM;
+        const int tok0 = tt * kPairTokens + (int)rank * (kPairTokens / 2);
+        for (int i = 0; i < kb; ++i, ++gi) {
+          if (gi >= p.stages && !(ok = mbar_wait(smem_u32(&hdr->empty[stage]), phase ^ 1u, a.status, kStatusProducerTimeout))) break;
+          const uint32_t full = smem_u32(&hdr->full[stage]);
+          // the first CTA's barrier counts the bytes of all four loads of the stage (two per CTA)
+          if (rank == 0) mbar_expect_tx(full, 2u * kPairStageBytes);
+          const uint32_t dst = stage0 + (uint32_t)stage * kPairStageBytes;
+          tma_load_2d_pair(dst, &map_w, full, 0, line0 + i * kTileN, hint_w);
+          tma_load_2d_pair(dst + a_bytes, &map_x, full, i * kTileK, tok0, hint_x);
+          if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+        }
       }
-      if (issued < n_it) {
+      if (!ok) {
         // a wait ran out: give the copies in flight a bounded time to land before the shared memory is given up
         const long long t0 = clock64();
         while (clock64() - t0 < 2000000LL) { }
@@ -598,37 +609,49 @@ gemm_wx_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
     // ===================== MMA issuer (first CTA of the pair only) =====================
     if (lane == 0 && rank == 0) {
       const uint32_t idesc = umma_idesc_bf16(kPairTokens, 256);
-      int stage = 0;
+      int stage = 0, r = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int i = 0; i < n_it; ++i) {
-        ok = mbar_wait(smem_u32(&hdr->full[stage]), phase, a.status, kStatusMmaTimeout);
+      for (int u = pair; u < n_units && ok; u += n_pairs, ++r) {
+        const int buf = r & 1;
+        // both CTAs' epilogues have drained this buffer (its first use passes at once)
+        ok = mbar_wait(smem_u32(&hdr->acc_empty[buf]), ((uint32_t)(r >> 1) & 1u) ^ 1u, a.status, kStatusMmaTimeout);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t sa = stage0 + (uint32_t)stage * kPairStageBytes;
-        const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sa + a_bytes);
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * kPairTokens);
+        for (int i = 0; i < kb; ++i) {
+          ok = mbar_wait(smem_u32(&hdr->full[stage]), phase, a.status, kStatusMmaTimeout);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t sa = stage0 + (uint32_t)stage * kPairStageBytes;
+          const uint64_t da = smem_desc_sw128(sa), db = smem_desc_sw128(sa + a_bytes);
 #pragma unroll
-        for (int k = 0; k < kTileK / 16; ++k)
-          umma_bf16_pair(tmem_base, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (i == 0 && k == 0) ? 0u : 1u);
-        umma_commit_pair(smem_u32(&hdr->empty[stage]));      // frees the stage in both CTAs when these MMAs retire
-        if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+          for (int k = 0; k < kTileK / 16; ++k)
+            umma_bf16_pair(d_tmem, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (i == 0 && k == 0) ? 0u : 1u);
+          umma_commit_pair(smem_u32(&hdr->empty[stage]));    // frees the stage in both CTAs when these MMAs retire
+          if (++stage == p.stages) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) umma_commit_pair(smem_u32(&hdr->acc_full[buf]));
       }
-      if (ok) umma_commit_pair(smem_u32(&hdr->acc_full[0]));
     }
   } else {
     // ===================== epilogue (4 warps, one TMEM lane quarter each): this CTA's 128 rows x 256 tokens ====
     pdl_wait();
     const int quarter = warp & 3;
     const int row = quarter * 32 + lane;
-    const int tok0 = tok_tile * kPairTokens;
-    int n_valid = a.n_tok - tok0;
-    if (n_valid > kPairTokens) n_valid = kPairTokens;
-    bool ok = mbar_wait(smem_u32(&hdr->acc_full[0]), 0u, a.status, kStatusEpilogueTimeout);
-    ok = __all_sync(0xffffffffu, ok);
-    if (ok) {
+    int r = 0;
+    for (int u = pair; u < n_units; u += n_pairs, ++r) {
+      const int wt = u / tok_tiles, tt = u - wt * tok_tiles;
+      const int buf = r & 1;
+      const int tok0 = tt * kPairTokens;
+      int n_valid = a.n_tok - tok0;
+      if (n_valid > kPairTokens) n_valid = kPairTokens;
+      bool ok = mbar_wait(smem_u32(&hdr->acc_full[buf]), (uint32_t)(r >> 1) & 1u, a.status, kStatusEpilogueTimeout);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
       tc_fence_after();
-      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16);
-      const int n = tile * kTileM + row;
+      const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * kPairTokens);
+      const int n = (2 * wt + (int)rank) * kTileM + row;
       if (a.mode == kGemmDirectF32) {
         for (int c = 0; c < kPairTokens; c += 32) {
           float v[32];
@@ -665,6 +688,13 @@ gemm_wx_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
           }
         }
       }
+      // the buffer may be overwritten once all eight epilogue warps of the pair have read it
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) {
+        if (rank == 0) mbar_arrive(smem_u32(&hdr->acc_empty[buf]));
+        else mbar_arrive_leader(smem_u32(&hdr->acc_empty[buf]));
+      }
     }
   }
 
@@ -674,7 +704,7 @@ gemm_wx_pair_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_cons
   cluster_sync_all();
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc_pair(tmem_base, (uint32_t)kPairTokens);
+    tmem_dealloc_pair(tmem_base, 2u * kPairTokens);
   }
 }
 

@@ -327,8 +327,10 @@ int run_gemm_pair(ss_ctx* c, const CUtensorMap& mw, const CUtensorMap& mx, int n
   a.out_f32 = out_f32;
   a.ld_out = ld_out;
   a.status = c->status;
-  SS_CUDA(c, launch(c, gemm_wx_pair_kernel, dim3(2 * ceil_div(n_tok, kPairTokens), a.p.n_tiles / 2), dim3(kGemmThreads),
-                    (size_t)a.p.smem_bytes, mw, mx, a));
+  a.p.gridy = ceil_div(n_tok, kPairTokens);                          // token tiles
+  const int n_units = (a.p.n_tiles / 2) * a.p.gridy;
+  a.p.gridx = std::min(n_units, c->n_sm / 2);                        // pairs of CTAs, each walking its units
+  SS_CUDA(c, launch(c, gemm_wx_pair_kernel, dim3(2 * a.p.gridx), dim3(kGemmThreads), (size_t)a.p.smem_bytes, mw, mx, a));
   return SS_OK;
 }
 
