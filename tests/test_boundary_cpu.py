@@ -35,6 +35,7 @@ def test_struct_sizes_match_header_layout():
     assert ctypes.sizeof(api.ss_batch_desc) == 16
     assert ctypes.sizeof(api.ss_batch_log) == 32
     assert ctypes.sizeof(api.ss_group_stats) == 64
+    assert ctypes.sizeof(api.ss_step_opts) == 32            # four pointers: forced tokens, logits, hidden, choice
 
 
 def test_strerror_and_argument_errors():
