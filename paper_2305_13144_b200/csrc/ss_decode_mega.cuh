@@ -127,6 +127,7 @@ struct MegaSmem {
   uint8_t active_s[kMaxBatch];     // rows active in this step
 };
 static_assert(sizeof(float) * 8 * 9 * 132 >= 2 * (2 * 4 * 64 * 4), "arg-max scratch aliases att_s");
+static_assert(sizeof(float) * 8 * 9 * 132 >= 8 * 32 * 36 * sizeof(float), "the drain's transposition scratch aliases att_s");
 
 __device__ __forceinline__ void named_bar_workers() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
@@ -1134,10 +1135,36 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
           for (int c = 0; c < 128; c += 64) {
             uint32_t v[64];
             tmem_ld64(taddr + c, v);
-            if (tok < a.B) {
+            if (a.NT <= 32) {
+              // few rows: the tail is a chain of latencies, the direct stores are the shortest one
+              if (tok < a.B) {
 #pragma unroll
-              for (int j = 0; j < 64; j += 4)
-                *reinterpret_cast<uint4*>(dst + c + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                for (int j = 0; j < 64; j += 4)
+                  *reinterpret_cast<uint4*>(dst + c + j) = make_uint4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+              }
+            } else {
+              // many rows: a lane holds one token's outputs, so direct 128-bit stores put every lane's 16 bytes
+              // into a sector of its own, 1 KiB apart, and the drain is bound by the sectors it writes.  The
+              // warp turns 32 outputs at a time through shared memory (rows padded to 36 floats: both
+              // directions free of bank conflicts) and stores whole 128-byte lines, four tokens per instruction.
+              float* tr = &sm->att_s[0][0][0] + wid * (32 * 36);
+              const int t_hi = lane >> 3, cg = lane & 7;
+#pragma unroll
+              for (int sub = 0; sub < 2; ++sub) {
+#pragma unroll
+                for (int j = 0; j < 32; j += 4)
+                  *reinterpret_cast<uint4*>(tr + lane * 36 + j) =
+                      make_uint4(v[sub * 32 + j], v[sub * 32 + j + 1], v[sub * 32 + j + 2], v[sub * 32 + j + 3]);
+                __syncwarp();
+                for (int i = 0; i < per_q / 4; ++i) {
+                  const int tl = 4 * i + t_hi;
+                  const int tg = mt * 128 + quarter * per_q + tl;
+                  if (tg < a.B)
+                    *reinterpret_cast<uint4*>(a.partial + (slot * a.NT + tg) * kTileN + colhalf * 128 + c + sub * 32 + 4 * cg) =
+                        *reinterpret_cast<const uint4*>(tr + tl * 36 + 4 * cg);
+                }
+                __syncwarp();
+              }
             }
           }
         }
