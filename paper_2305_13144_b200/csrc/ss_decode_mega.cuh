@@ -1135,8 +1135,8 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
           for (int c = 0; c < 128; c += 64) {
             uint32_t v[64];
             tmem_ld64(taddr + c, v);
-            if (a.NT <= 32) {
-              // few rows: the tail is a chain of latencies, the direct stores are the shortest one
+            if (a.NT <= 16) {
+              // one MMA's worth of rows or fewer: the tail is a chain of latencies, direct stores are the shortest one
               if (tok < a.B) {
 #pragma unroll
                 for (int j = 0; j < 64; j += 4)
