@@ -120,8 +120,8 @@ struct MegaSmem {
   int pair_id[8], pair_ustart[9], pair_n, pair_next, pair_lo, pair_hi;
   // per-step attention set-up that does not change from layer to layer (valid when att_single)
   int att_single;                  // the CTA's pairs fit one pass: the lists above are built once per step
-  int pair_pos[8], pair_pgnew[8];  // new token's position and page
-  int unit_pg[8][8];               // page ids of each warp's units (when it has at most 8)
+  int pair_pos[8], pair_pgnew[8];  // per pass: new token's position and page
+  int unit_pg[8][8];               // per pass: ids of the first 8 pages of each warp's slice of the scan
   float rope_c[8][128], rope_sn[8][128];   // cos / sin of the new position per pair, cooperative lane layout
   int4 seg_tab[kSegTabEntries];    // tile tables of the per-layer projections (when they fit)
   uint8_t active_s[kMaxBatch];     // rows active in this step
@@ -385,6 +385,51 @@ constexpr int kAttnPass = 8;               // pairs per pass (= worker warps)
 constexpr int kAttnU = 2;                  // load steps per work unit of the cache scan (one batch of loads in flight)
 constexpr int kAttnSlots = 9;              // partials per pair: one per warp + the new token
 
+// Tables of the pass whose pair list is in shared memory: the new tokens' positions and pages, the ids of the first
+// pages of every warp's slice of the scan (all requested together, so that the scan itself starts no chain of
+// dependent look-ups), and -- with_rope, for a CTA whose pairs fit one pass: once per step -- the rotations.
+template <int DH>
+__device__ __forceinline__ void attention_pass_tables(const MegaArgs& a, MegaSmem* sm, int wtid, bool with_rope) {
+  constexpr int EPL = DH / 32;
+  constexpr int UT = kAttnU * (32 / (DH / 32));
+  constexpr int UPP = kPageTokens / UT;
+  const int lane = wtid & 31, wid = wtid >> 5;
+  const int H = a.H;
+  const int np = sm->pair_n, U = sm->pair_ustart[np];
+  if (wid < np) {
+    const int p = sm->pair_id[wid];
+    const int r = p / H;
+    const int pos = a.st.ctx_len[r];
+    if (with_rope) {
+#pragma unroll
+      for (int j = 0; j < EPL; ++j) {
+        float sn, cs;
+        sincosf((float)pos * a.inv_freq[(lane & 15) * EPL + j], &sn, &cs);
+        sm->rope_c[wid][lane * EPL + j] = cs;
+        sm->rope_sn[wid][lane * EPL + j] = sn;
+      }
+    }
+    if (lane == 0) {
+      sm->pair_pos[wid] = pos;
+      sm->pair_pgnew[wid] = a.st.block_table[(size_t)r * a.st.max_pages + pos / kPageTokens];
+    }
+  }
+  // page ids of the first (up to 8) distinct pages of this warp's slice, in scan order
+  const int u0 = (int)((long long)wid * U / 8), u1 = (int)((long long)(wid + 1) * U / 8);
+  const int u = u0 + lane;
+  int j = 0, ui = 0;
+  bool newpage = false;
+  if (u < u1) {
+    while (j + 1 < np && sm->pair_ustart[j + 1] <= u) ++j;
+    ui = u - sm->pair_ustart[j];
+    newpage = lane == 0 || ui % UPP == 0;
+  }
+  const unsigned int starts = __ballot_sync(0xffffffffu, newpage);
+  const int ord = __popc(starts & (0xffffffffu >> (31 - lane))) - 1;
+  if (newpage && ord < 8)
+    sm->unit_pg[wid][ord] = a.st.block_table[(size_t)(sm->pair_id[j] / H) * a.st.max_pages + ui / UPP];
+}
+
 // Once per step (the lengths do not change between layers): units per row, this CTA's run of pairs, and --
 // when the run fits one pass -- the pass list, the new tokens' positions/pages/rotations and the ids of
 // the first pages of every warp's slice.
@@ -465,39 +510,7 @@ __device__ void attention_setup(const MegaArgs& a, MegaSmem* sm, int wtid) {
     if (lane == 0) { sm->pair_n = n; sm->pair_next = p; sm->pair_ustart[n] = ustart; sm->att_single = more ? 0 : 1; }
   }
   named_bar_workers();
-  if (sm->att_single) {
-    const int np = sm->pair_n, U = sm->pair_ustart[np];
-    if (wid < np) {
-      const int p = sm->pair_id[wid];
-      const int r = p / H;
-      const int pos = a.st.ctx_len[r];
-#pragma unroll
-      for (int j = 0; j < EPL; ++j) {
-        float sn, cs;
-        sincosf((float)pos * a.inv_freq[(lane & 15) * EPL + j], &sn, &cs);
-        sm->rope_c[wid][lane * EPL + j] = cs;
-        sm->rope_sn[wid][lane * EPL + j] = sn;
-      }
-      if (lane == 0) {
-        sm->pair_pos[wid] = pos;
-        sm->pair_pgnew[wid] = a.st.block_table[(size_t)r * a.st.max_pages + pos / kPageTokens];
-      }
-    }
-    // page ids of the first (up to 8) distinct pages of this warp's slice, in scan order
-    const int u0 = (int)((long long)wid * U / 8), u1 = (int)((long long)(wid + 1) * U / 8);
-    const int u = u0 + lane;
-    int j = 0, ui = 0;
-    bool newpage = false;
-    if (u < u1) {
-      while (j + 1 < np && sm->pair_ustart[j + 1] <= u) ++j;
-      ui = u - sm->pair_ustart[j];
-      newpage = lane == 0 || ui % UPP == 0;
-    }
-    const unsigned int starts = __ballot_sync(0xffffffffu, newpage);
-    const int ord = __popc(starts & (0xffffffffu >> (31 - lane))) - 1;
-    if (newpage && ord < 8)
-      sm->unit_pg[wid][ord] = a.st.block_table[(size_t)(sm->pair_id[j] / H) * a.st.max_pages + ui / UPP];
-  }
+  if (sm->att_single) attention_pass_tables<DH>(a, sm, wtid, true);
   named_bar_workers();
 }
 
@@ -537,6 +550,11 @@ __device__ void stage_attention(const MegaArgs& a, MegaSmem* sm, int wtid, int l
     }
     for (int i = wtid; i < kAttnPass * kAttnSlots; i += kMegaWorkers) sm->att_s[i / kAttnSlots][i % kAttnSlots][DH] = -CUDART_INF_F;
     named_bar_workers();
+    if (!single) {
+      // positions and page ids of this pass, looked up together (a CTA with one pass did this once per step)
+      attention_pass_tables<DH>(a, sm, wtid, false);
+      named_bar_workers();
+    }
     const int np_pass = sm->pair_n;
     const int U_pass = sm->pair_ustart[np_pass];
 
@@ -544,7 +562,7 @@ __device__ void stage_attention(const MegaArgs& a, MegaSmem* sm, int wtid, int l
     if (wid < np_pass) {
       const int p = sm->pair_id[wid];
       const int r = p / H, hd = p - r * H;
-      const int pos = single ? sm->pair_pos[wid] : a.st.ctx_len[r];
+      const int pos = sm->pair_pos[wid];
       const float inv = warp_row_inv_rms(a, r, lane);
       const int e0 = lane * EPL;
       float sn[EPL], cs[EPL];
@@ -565,7 +583,7 @@ __device__ void stage_attention(const MegaArgs& a, MegaSmem* sm, int wtid, int l
         partials_sum<EPL, 4>(a.partial, gs, a.NT, tk, nk, r, lk, kx);
         partials_sum<EPL, 4>(a.partial, gs, a.NT, tv, nv, r, lv, vx);
       }
-      int pg = single ? sm->pair_pgnew[wid] : a.st.block_table[(size_t)r * a.st.max_pages + pos / kPageTokens];
+      int pg = sm->pair_pgnew[wid];
       if (pg < 0 || pg >= a.kv.n_pages) { atomicCAS(a.status, 0u, (uint32_t)kStatusBadPage); pg = -1; }
       bf16* kdst = a.kv.pool + (size_t)layer * a.kv.layer_stride + (size_t)(pg < 0 ? 0 : pg) * a.kv.page_elems +
                    ((size_t)hd * kPageTokens + (pos % kPageTokens)) * DH + e0;
@@ -635,10 +653,10 @@ __device__ void stage_attention(const MegaArgs& a, MegaSmem* sm, int wtid, int l
         const int r = p / H, hd = p - r * H;
         const int ui = u - sm->pair_ustart[j];           // unit of the pair: page ui / UPP, batch ui % UPP of it
         const int pi = ui / UPP;
-        const int pos = single ? sm->pair_pos[j] : a.st.ctx_len[r];
+        const int pos = sm->pair_pos[j];
         if (u == u0 || ui % UPP == 0) {
           ++kpage;
-          pg = (single && kpage < 8) ? sm->unit_pg[wid][kpage] : a.st.block_table[(size_t)r * a.st.max_pages + pi];
+          pg = kpage < 8 ? sm->unit_pg[wid][kpage] : a.st.block_table[(size_t)r * a.st.max_pages + pi];
           if (pg < 0 || pg >= a.kv.n_pages) { atomicCAS(a.status, 0u, (uint32_t)kStatusBadPage); pg = 0; }
         }
         const int tcount = min(kPageTokens, pos - pi * kPageTokens);
