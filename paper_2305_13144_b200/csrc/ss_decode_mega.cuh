@@ -120,6 +120,7 @@ struct MegaSmem {
   int pair_id[8], pair_ustart[9], pair_n, pair_next, pair_lo, pair_hi;
   // per-step attention set-up that does not change from layer to layer (valid when att_single)
   int att_single;                  // the CTA's pairs fit one pass: the lists above are built once per step
+  int att_warp_pairs;              // the CTA's run has many pairs: every warp takes whole pairs (attention_warp_pairs)
   int pair_pos[8], pair_pgnew[8];  // per pass: new token's position and page
   int unit_pg[8][8];               // per pass: ids of the first 8 pages of each warp's slice of the scan
   float rope_c[8][128], rope_sn[8][128];   // cos / sin of the new position per pair, cooperative lane layout
@@ -384,6 +385,7 @@ __device__ __forceinline__ void group_bar(int id, int threads) {
 constexpr int kAttnPass = 8;               // pairs per pass (= worker warps)
 constexpr int kAttnU = 2;                  // load steps per work unit of the cache scan (one batch of loads in flight)
 constexpr int kAttnSlots = 9;              // partials per pair: one per warp + the new token
+constexpr int kAttnWarpPairsMin = 24;      // pairs in a CTA's run from which every warp takes whole pairs (at most 1/3 idle)
 
 // Tables of the pass whose pair list is in shared memory: the new tokens' positions and pages, the ids of the first
 // pages of every warp's slice of the scan (all requested together, so that the scan itself starts no chain of
@@ -433,11 +435,9 @@ __device__ __forceinline__ void attention_pass_tables(const MegaArgs& a, MegaSme
 // Once per step (the lengths do not change between layers): units per row, this CTA's run of pairs, and --
 // when the run fits one pass -- the pass list, the new tokens' positions/pages/rotations and the ids of
 // the first pages of every warp's slice.
-template <int DH>
+template <int DH, bool WIDE>
 __device__ void attention_setup(const MegaArgs& a, MegaSmem* sm, int wtid) {
-  constexpr int EPL = DH / 32;
   constexpr int UT = kAttnU * (32 / (DH / 32));   // cached tokens per work unit (16 at Dh 128, 32 at Dh 64)
-  constexpr int UPP = kPageTokens / UT;           // units per page
   const int lane = wtid & 31, wid = wtid >> 5;
   const int H = a.H, B = a.B;
   // ---- per-step copies in shared memory: which rows are active, and the per-layer tile tables
@@ -508,10 +508,256 @@ __device__ void attention_setup(const MegaArgs& a, MegaSmem* sm, int wtid) {
       if (sm->prefix[r + 1] - sm->prefix[r] > 0) more = true; else q = (r + 1) * H;
     }
     if (lane == 0) { sm->pair_n = n; sm->pair_next = p; sm->pair_ustart[n] = ustart; sm->att_single = more ? 0 : 1; }
+    if constexpr (WIDE) {
+      // pairs with work in the whole run
+      int cnt = 0;
+      for (int q = p_begin; q < p_end; ) {
+        const int r = q / H;
+        const int e = min(p_end, (r + 1) * H);
+        if (sm->prefix[r + 1] - sm->prefix[r] > 0) cnt += e - q;
+        q = e;
+      }
+      if (lane == 0) sm->att_warp_pairs = cnt >= kAttnWarpPairsMin ? 1 : 0;
+    }
   }
   named_bar_workers();
   if (sm->att_single) attention_pass_tables<DH>(a, sm, wtid, true);
   named_bar_workers();
+}
+
+// ---- pieces of the attention stage, each run by one warp, as attention_warp_pairs puts them together ----------
+// (stage_attention below has the same steps written out in place: it is the path of the small batches, and its
+// register allocation is what the whole kernel's speed hangs on)
+template <int DH> struct AttnLayout {
+  static constexpr int GROUP = DH / 32;           // lanes per key in the cache scan
+  static constexpr int KPW = 32 / GROUP;          // keys per warp-wide load step
+  static constexpr int EPL = DH / 32;             // cooperative layout: consecutive dimensions per lane
+  static constexpr int U = kAttnU;                // load steps per work unit: one batch of loads
+  static constexpr int UPP = kPageTokens / (U * KPW);   // units per page (2 at Dh 128, 1 at Dh 64)
+};
+
+// A: the pair's rotated, scaled query into qs[DH]; the new token's k, v appended to page pg at position pos and
+// entered as the partial ns[DH + 2] = (v, score, 1).  cs / sn: the rotation of this lane's dimensions.
+template <int DH>
+__device__ __forceinline__ void attn_prepare_pair(const MegaArgs& a, const MegaSmem* sm, int layer, int lane, int r, int hd, int pos,
+                                                  int pg, const float (&cs)[DH / 32], const float (&sn)[DH / 32], float* qs, float* ns) {
+  constexpr int EPL = AttnLayout<DH>::EPL;
+  const int H = a.H, d = a.d;
+  const MegaGemmShape& gs = a.shape[0];
+  const float qscale = rsqrtf((float)DH) * 1.4426950408889634f;
+  const size_t v_off = (size_t)H * kPageTokens * DH;
+  const float inv = warp_row_inv_rms(a, r, lane);
+  const int e0 = lane * EPL;
+  float qx[EPL], kx[EPL], vx[EPL];
+  {
+    const int nq = hd * DH + e0, nk = d + nq, nv = 2 * d + nq;
+    const int4 tq = tile_seg(sm, gs, nq), tk = tile_seg(sm, gs, nk), tv = tile_seg(sm, gs, nv);
+    PartialLoads<EPL, 4> lq, lk, lv;
+    partials_issue<EPL, 4>(a.partial, gs, a.NT, tq, nq, r, lq);
+    partials_issue<EPL, 4>(a.partial, gs, a.NT, tk, nk, r, lk);
+    partials_issue<EPL, 4>(a.partial, gs, a.NT, tv, nv, r, lv);
+    partials_sum<EPL, 4>(a.partial, gs, a.NT, tq, nq, r, lq, qx);
+    partials_sum<EPL, 4>(a.partial, gs, a.NT, tk, nk, r, lk, kx);
+    partials_sum<EPL, 4>(a.partial, gs, a.NT, tv, nv, r, lv, vx);
+  }
+  if (pg < 0 || pg >= a.kv.n_pages) { atomicCAS(a.status, 0u, (uint32_t)kStatusBadPage); pg = -1; }
+  bf16* kdst = a.kv.pool + (size_t)layer * a.kv.layer_stride + (size_t)(pg < 0 ? 0 : pg) * a.kv.page_elems +
+               ((size_t)hd * kPageTokens + (pos % kPageTokens)) * DH + e0;
+  float dot = 0.f;
+#pragma unroll
+  for (int j = 0; j < EPL; ++j) {
+    const float xq = qx[j] * inv, xk = kx[j] * inv;
+    const float pq = __shfl_xor_sync(0xffffffffu, xq, 16), pk = __shfl_xor_sync(0xffffffffu, xk, 16);
+    const float oq = (lane < 16) ? xq * cs[j] - pq * sn[j] : xq * cs[j] + pq * sn[j];
+    const float ok = (lane < 16) ? xk * cs[j] - pk * sn[j] : xk * cs[j] + pk * sn[j];
+    const float qf = oq * qscale;                     // the query is only ever an ALU operand: it stays fp32
+    const bf16 kb16 = __float2bfloat16_rn(ok), vb16 = __float2bfloat16_rn(vx[j] * inv);
+    if (pg >= 0) { kdst[j] = kb16; kdst[v_off + j] = vb16; }
+    qs[e0 + j] = qf;
+    ns[e0 + j] = __bfloat162float(vb16);
+    dot += qf * __bfloat162float(kb16);
+  }
+  dot = warp_sum(dot);
+  if (lane == 0) { ns[DH] = dot; ns[DH + 1] = 1.f; }
+}
+
+// B: one unit (U load steps of KPW keys; kb = first key of the page's head, s0 = first load step, tcount = the
+// page's tokens) folded into the running (m, l, acc) of the lane's key slot.
+template <int DH>
+__device__ __forceinline__ void attn_scan_unit(const bf16* __restrict__ kb, size_t v_off, int s0, int tcount, const float* qs, int g, int gl,
+                                               float& m, float& l, float (&acc)[32]) {
+  constexpr int GROUP = AttnLayout<DH>::GROUP, KPW = AttnLayout<DH>::KPW, U = AttnLayout<DH>::U;
+  uint4 kk[U][4], vv[U][4];
+#pragma unroll
+  for (int uu = 0; uu < U; ++uu) {
+    const int t = (s0 + uu) * KPW + g;
+    if (t < tcount) {
+      const uint4* kp = reinterpret_cast<const uint4*>(kb + (size_t)t * DH);
+      const uint4* vp = reinterpret_cast<const uint4*>(kb + (size_t)t * DH + v_off);
+#pragma unroll
+      for (int c = 0; c < 4; ++c) { kk[uu][c] = __ldg(kp + c * GROUP + gl); vv[uu][c] = __ldg(vp + c * GROUP + gl); }
+    } else {
+#pragma unroll
+      for (int c = 0; c < 4; ++c) { kk[uu][c] = make_uint4(0, 0, 0, 0); vv[uu][c] = kk[uu][c]; }
+    }
+  }
+  float sc_[U];
+#pragma unroll
+  for (int uu = 0; uu < U; ++uu) {
+    float dot = 0.f;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      float kf[8];
+      unpack8(kk[uu][c], kf);
+      const float4 qa = *reinterpret_cast<const float4*>(qs + (c * GROUP + gl) * 8);
+      const float4 qb = *reinterpret_cast<const float4*>(qs + (c * GROUP + gl) * 8 + 4);
+      dot += qa.x * kf[0] + qa.y * kf[1] + qa.z * kf[2] + qa.w * kf[3] + qb.x * kf[4] + qb.y * kf[5] +
+             qb.z * kf[6] + qb.w * kf[7];
+    }
+#pragma unroll
+    for (int o = GROUP / 2; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+    sc_[uu] = ((s0 + uu) * KPW + g < tcount) ? dot : -CUDART_INF_F;
+  }
+  float mn = m;
+#pragma unroll
+  for (int uu = 0; uu < U; ++uu) mn = fmaxf(mn, sc_[uu]);
+  if (mn != -CUDART_INF_F) {
+    if (mn != m) {
+      const float sc = exp2f(m - mn);
+      l *= sc;
+#pragma unroll
+      for (int e = 0; e < 32; ++e) acc[e] *= sc;
+      m = mn;
+    }
+#pragma unroll
+    for (int uu = 0; uu < U; ++uu) {
+      if (sc_[uu] != -CUDART_INF_F) {
+        const float pw = exp2f(sc_[uu] - mn);
+        l += pw;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+          float vf[8];
+          unpack8(vv[uu][c], vf);
+#pragma unroll
+          for (int e = 0; e < 8; ++e) acc[c * 8 + e] += pw * vf[e];
+        }
+      }
+    }
+  }
+}
+
+// The warp's KPW key slots merged, the result stored as the partial slot[DH + 2] = (acc, m, l); (m, l, acc) reset.
+template <int DH>
+__device__ __forceinline__ void attn_flush(float* slot, int g, int gl, float& m, float& l, float (&acc)[32]) {
+  constexpr int GROUP = AttnLayout<DH>::GROUP;
+#pragma unroll
+  for (int o = GROUP; o < 32; o <<= 1) {
+    const float om = __shfl_xor_sync(0xffffffffu, m, o);
+    const float ol = __shfl_xor_sync(0xffffffffu, l, o);
+    const float mn = fmaxf(m, om);
+    const float w0 = (m == -CUDART_INF_F) ? 0.f : exp2f(m - mn);
+    const float w1 = (om == -CUDART_INF_F) ? 0.f : exp2f(om - mn);
+    l = l * w0 + ol * w1;
+#pragma unroll
+    for (int e = 0; e < 32; ++e) {
+      const float oa = __shfl_xor_sync(0xffffffffu, acc[e], o);
+      acc[e] = acc[e] * w0 + oa * w1;
+    }
+    m = mn;
+  }
+  if (g == 0) {
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+#pragma unroll
+      for (int e = 0; e < 8; ++e) slot[(c * GROUP + gl) * 8 + e] = acc[c * 8 + e];
+    if (gl == 0) { slot[DH] = m; slot[DH + 1] = l; }
+  }
+  m = -CUDART_INF_F;
+  l = 0.f;
+#pragma unroll
+  for (int e = 0; e < 32; ++e) acc[e] = 0.f;
+}
+
+// C: the pair's partials slots[0 .. kAttnSlots) merged and written as bf16 output of (row r, head hd).
+template <int DH>
+__device__ __forceinline__ void attn_merge_pair(const MegaArgs& a, const float (*slots)[132], int lane, int r, int hd) {
+  constexpr int EPL = AttnLayout<DH>::EPL;
+  const int e0 = lane * EPL;
+  float M = -CUDART_INF_F;
+  for (int k = 0; k < kAttnSlots; ++k) M = fmaxf(M, slots[k][DH]);
+  float L = 0.f, A[EPL];
+#pragma unroll
+  for (int j = 0; j < EPL; ++j) A[j] = 0.f;
+  for (int k = 0; k < kAttnSlots; ++k) {
+    const float mk = slots[k][DH];
+    if (mk == -CUDART_INF_F) continue;
+    const float wt = exp2f(mk - M);
+    L += slots[k][DH + 1] * wt;
+#pragma unroll
+    for (int j = 0; j < EPL; ++j) A[j] += slots[k][e0 + j] * wt;
+  }
+  const float il = 1.f / L;
+#pragma unroll
+  for (int j = 0; j < EPL; ++j) a.o[(size_t)r * a.d + hd * DH + e0 + j] = __float2bfloat16_rn(A[j] * il);
+}
+
+// Wide batches, where a CTA's run has many pairs: every warp takes whole pairs (the run's pairs with work, in turn)
+// and does all three steps for them by itself, so nothing is shared between the warps and nothing holds them in
+// step: while one warp builds a query, the others' loads are in flight.  The pair's page ids are looked up by the
+// lanes together (lane i: pages i and i + 32) and handed out by shuffle.
+template <int DH>
+__device__ void attention_warp_pairs(const MegaArgs& a, MegaSmem* sm, int wtid, int layer) {
+  using L = AttnLayout<DH>;
+  constexpr int GROUP = L::GROUP, EPL = L::EPL, U = L::U, UPP = L::UPP;
+  const int lane = wtid & 31, wid = wtid >> 5;
+  const int gl = lane % GROUP, g = lane / GROUP;
+  const int H = a.H;
+  const bf16* kv_layer = a.kv.pool + (size_t)layer * a.kv.layer_stride;
+  const size_t v_off = (size_t)H * kPageTokens * DH;
+  const int p_begin = sm->pair_lo, p_end = sm->pair_hi + 1;
+  float (*slots)[132] = sm->att_s[wid];
+  float* qs = sm->q_s[wid];
+  int n = 0;
+  for (int p = p_begin; p < p_end; ) {
+    const int r = p / H;
+    const int npr = sm->prefix[r + 1] - sm->prefix[r];
+    if (npr <= 0) { p = (r + 1) * H; continue; }
+    if ((n++ & 7) != wid) { ++p; continue; }
+    const int hd = p - r * H;
+    const int pos = a.st.ctx_len[r];
+    const int last_page = pos / kPageTokens;            // the new token's page
+    const int32_t* bt = a.st.block_table + (size_t)r * a.st.max_pages;
+    const int pgs0 = lane <= last_page ? bt[lane] : 0;
+    const int pgs1 = lane + 32 <= last_page ? bt[lane + 32] : 0;
+    if (lane < kAttnSlots) slots[lane][DH] = -CUDART_INF_F;
+    float sn[EPL], cs[EPL];
+#pragma unroll
+    for (int j = 0; j < EPL; ++j) sincosf((float)pos * a.inv_freq[(lane & 15) * EPL + j], &sn[j], &cs[j]);
+    const int pg_new = last_page < 32 ? __shfl_sync(0xffffffffu, pgs0, last_page)
+                                      : (last_page < 64 ? __shfl_sync(0xffffffffu, pgs1, last_page - 32) : bt[last_page]);
+    __syncwarp();
+    attn_prepare_pair<DH>(a, sm, layer, lane, r, hd, pos, pg_new, cs, sn, qs, slots[kAttnSlots - 1]);
+    __syncwarp();
+    float m = -CUDART_INF_F, l = 0.f, acc[32];
+#pragma unroll
+    for (int e = 0; e < 32; ++e) acc[e] = 0.f;
+    int pg = 0;
+    for (int ui = 0; ui < npr; ++ui) {
+      const int pi = ui / UPP;
+      if (ui % UPP == 0) {
+        pg = pi < 32 ? __shfl_sync(0xffffffffu, pgs0, pi) : (pi < 64 ? __shfl_sync(0xffffffffu, pgs1, pi - 32) : bt[pi]);
+        if (pg < 0 || pg >= a.kv.n_pages) { atomicCAS(a.status, 0u, (uint32_t)kStatusBadPage); pg = 0; }
+      }
+      const int tcount = min(kPageTokens, pos - pi * kPageTokens);
+      const bf16* kb = kv_layer + (size_t)pg * a.kv.page_elems + (size_t)hd * kPageTokens * DH;
+      attn_scan_unit<DH>(kb, v_off, (ui % UPP) * U, tcount, qs, g, gl, m, l, acc);
+    }
+    attn_flush<DH>(slots[0], g, gl, m, l, acc);
+    __syncwarp();
+    attn_merge_pair<DH>(a, slots, lane, r, hd);
+    __syncwarp();
+    ++p;
+  }
 }
 
 template <int DH>
@@ -919,7 +1165,10 @@ __device__ void stage_final(const MegaArgs& a, int wtid) {
 }
 
 // ------------------------------------------------------------------------------------ the kernel
-template <int DH>
+// WIDE: the variant for batches of more than 64 rows, which adds attention_warp_pairs.  It is an instantiation of
+// its own because the batches up to 64 rows live on this kernel's register allocation: the same code with the
+// extra path compiled in ran the 16-row step 2.5 % slower.
+template <int DH, bool WIDE>
 __global__ void __launch_bounds__(kMegaThreads, 1)
 decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_o,
                         const __grid_constant__ CUtensorMap map_act, const __grid_constant__ MegaArgs a) {
@@ -1114,7 +1363,7 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
     int tr = 0;
     if (tracer) a.trace[tr++] = global_timer_ns();
     if (cta == 0 && wtid == 0) a.st.scalars[1] = 0;   // rows still active after this step (counted in the last stage)
-    attention_setup<DH>(a, sm, wtid);
+    attention_setup<DH, WIDE>(a, sm, wtid);
     stage_residual(a, sm, wtid, 0, nullptr, a.norm_ptr[0], a.n_layers == 0);
     ok = grid_barrier(a, sm, epoch, wtid, true);
     if (ok && wtid == 0) { __threadfence_block(); sm->act_epoch = 1; }
@@ -1200,7 +1449,12 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
       if (tracer) a.trace[tr++] = global_timer_ns();       // every CTA's partials visible
       // ---- the stage that consumes the projection
       if (type == 0) {
-        stage_attention<DH>(a, sm, wtid, layer);
+        if constexpr (WIDE) {
+          if (sm->att_warp_pairs) attention_warp_pairs<DH>(a, sm, wtid, layer);
+          else stage_attention<DH>(a, sm, wtid, layer);
+        } else {
+          stage_attention<DH>(a, sm, wtid, layer);
+        }
       } else if (type == 1) {
         stage_residual(a, sm, wtid, 1, &a.shape[1], a.norm_ptr[2 * layer + 1], false);
       } else if (type == 2) {

@@ -550,7 +550,10 @@ int enqueue_decode_step(ss_ctx* c, const ss_step_opts* opts, int32_t* next_token
   a.trace = c->trace_on ? c->trace : nullptr;
   a.wait_limit = c->wait_limit;
   void* args[4] = {(void*)mx, (void*)mo, (void*)ma, (void*)&a};
-  const void* fn = m.head_dim == 128 ? (const void*)decode_step_mega_kernel<128> : (const void*)decode_step_mega_kernel<64>;
+  const bool wide = NT > 64;
+  const void* fn = m.head_dim == 128
+                       ? (wide ? (const void*)decode_step_mega_kernel<128, true> : (const void*)decode_step_mega_kernel<128, false>)
+                       : (wide ? (const void*)decode_step_mega_kernel<64, true> : (const void*)decode_step_mega_kernel<64, false>);
   SS_CUDA(c, cudaLaunchCooperativeKernel(fn, dim3(c->n_sm), dim3(kMegaThreads), args, smem, c->stream));
   c->grid_epochs += 1 + 2 * (unsigned long long)(4 * m.n_layers + 1);
   c->launches++;
@@ -792,9 +795,13 @@ int ss_create(const ss_model_cfg* model, const ss_runtime_cfg* rt, void* dev_are
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(gemm_wx_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(decode_step_mega_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    e = cudaFuncSetAttribute(decode_step_mega_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(decode_step_mega_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    e = cudaFuncSetAttribute(decode_step_mega_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(decode_step_mega_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e == cudaSuccess)
+    e = cudaFuncSetAttribute(decode_step_mega_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e != cudaSuccess) {
     c->last_cuda = (int)e;
     delete c;
