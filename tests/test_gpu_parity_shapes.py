@@ -60,9 +60,31 @@ def test_13b_shape_two_layers_batch16():
     assert el <= large_shape_tol(2) and eh <= large_shape_tol(2), (el, eh)
 
 
+@pytest.mark.parametrize("B", [48, 80])
+def test_13b_shape_two_layers_attention_in_several_passes(B):
+    """40 heads x 48 or 80 rows are 13 or 22 (row, head) pairs per CTA of a 148-SM part: more than the eight of one
+    pass, fewer than the 24 from which every warp takes whole pairs.  48 rows run in the kernel of the batches up
+    to 64 rows, 80 rows in the one for wide batches; prompts of 20 to 90 tokens, so rows differ in pages; two of
+    the followed rows end early."""
+    shape = synth.LLAMA_13B.with_layers(2)
+    w = synth.make_weights(shape, seed=13)
+    rng = np.random.default_rng(1000 + B)
+    cap = 3
+    lens = rng.integers(20, 91, size=B)
+    prompts = [rng.integers(3, shape.vocab, size=int(n)).tolist() for n in lens]
+    targets = rng.integers(2, 6, size=B).astype(np.int32)
+    follow = [0, B // 3, B // 2, B - 1]
+    targets[follow[1]], targets[follow[2]] = 1, 2
+    el, eh, steps = teacher_forced(shape, w, prompts, targets, cap, follow=follow, dtype=np.float32,
+                                   max_batch=128, max_ctx=128, max_prefill=8192, max_new=8, kv_tokens=128 * 128)
+    assert steps == cap
+    assert el <= large_shape_tol(2) and eh <= large_shape_tol(2), (el, eh)
+
+
 def test_13b_shape_two_layers_wide_batch():
     """The variable-batch-size arm's launch configuration at the 13B shape: 136 rows (two 128-lane token
-    tiles, the second with 8 rows), short prompts; the oracle follows six rows spread over both tiles."""
+    tiles, the second with 8 rows), short prompts; the oracle follows six rows spread over both tiles.  A CTA's run
+    has about 37 pairs here, so every warp takes whole pairs."""
     shape = synth.LLAMA_13B.with_layers(2)
     w = synth.make_weights(shape, seed=13)
     rng = np.random.default_rng(136)
@@ -74,5 +96,24 @@ def test_13b_shape_two_layers_wide_batch():
     targets[63], targets[128] = 2, 4
     el, eh, steps = teacher_forced(shape, w, prompts, targets, cap, follow=follow, dtype=np.float32,
                                    max_batch=256, max_ctx=128, max_prefill=8192, max_new=8, kv_tokens=256 * 64)
+    assert steps == cap
+    assert el <= large_shape_tol(2) and eh <= large_shape_tol(2), (el, eh)
+
+
+def test_many_heads_long_contexts_pages_beyond_the_first_64():
+    """A one-layer decoder with 32 heads x 64 and 120 rows whose prompts all have 2050 to 2110 tokens: 26 (row,
+    head) pairs per CTA, so every warp takes whole pairs, and 65 or 66 pages per row, so the scan goes through the
+    page ids a warp's lanes hold (pages 0..31 and 32..63) and the ones it looks up one by one beyond them."""
+    shape = synth.ModelShape(n_layers=1, d_model=2048, n_heads=32, head_dim=64, d_ffn=512, vocab=1024)
+    w = synth.make_weights(shape, seed=21)
+    rng = np.random.default_rng(2100)
+    B, cap = 120, 3
+    lens = rng.integers(2050, 2111, size=B)
+    prompts = [rng.integers(3, shape.vocab, size=int(n)).tolist() for n in lens]
+    targets = rng.integers(2, 6, size=B).astype(np.int32)
+    follow = [0, 59, 119]
+    targets[59] = 2
+    el, eh, steps = teacher_forced(shape, w, prompts, targets, cap, follow=follow, dtype=np.float32,
+                                   max_batch=128, max_ctx=2176, max_prefill=8192, max_new=8, kv_tokens=128 * 2176)
     assert steps == cap
     assert el <= large_shape_tol(2) and eh <= large_shape_tol(2), (el, eh)
