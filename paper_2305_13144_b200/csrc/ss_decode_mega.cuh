@@ -769,7 +769,7 @@ __device__ void stage_attention(const MegaArgs& a, MegaSmem* sm, int wtid, int l
   constexpr int UPP = kPageTokens / (U * KPW);   // units per page (2 at Dh 128, 1 at Dh 64)
   const int lane = wtid & 31, wid = wtid >> 5;
   const int gl = lane % GROUP, g = lane / GROUP;
-  const int H = a.H, d = a.d, B = a.B;
+  const int H = a.H, d = a.d;
   const MegaGemmShape& gs = a.shape[0];
   const float qscale = rsqrtf((float)DH) * 1.4426950408889634f;
   const bf16* kv_layer = a.kv.pool + (size_t)layer * a.kv.layer_stride;
@@ -1175,7 +1175,7 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   MegaSmem* sm = reinterpret_cast<MegaSmem*>(smem_raw);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int cta = blockIdx.x, G = gridDim.x;
+  const int cta = blockIdx.x;
   const uint32_t stage0 = (smem_u32(smem_raw) + (uint32_t)sizeof(MegaSmem) + 1023u) & ~1023u;
   // ring: S activation blocks first, then S weight blocks.  A token tile shorter than 128 rows is read
   // by the tensor core as 128 rows anyway; the surplus rows fall on the blocks that follow.
