@@ -1179,12 +1179,14 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
   const uint32_t stage0 = (smem_u32(smem_raw) + (uint32_t)sizeof(MegaSmem) + 1023u) & ~1023u;
   // ring: S activation blocks first, then S weight blocks.  A token tile shorter than 128 rows is read
   // by the tensor core as 128 rows anyway; the surplus rows fall on the blocks that follow.
+  // the batches up to 64 rows always have one token tile, computed with the 64-lane instruction
+  const int m_tiles = WIDE ? a.m_tiles : 1;
   const uint32_t x_tile_bytes = (uint32_t)a.x_rows * kTileK * 2;
-  const uint32_t x_bytes = (uint32_t)a.m_tiles * x_tile_bytes;
+  const uint32_t x_bytes = (uint32_t)m_tiles * x_tile_bytes;
   const uint32_t stage_tx = (uint32_t)kBlockBytes + x_bytes;
   const int S = a.stages;
   const uint32_t x0 = stage0, w0 = stage0 + (uint32_t)S * x_bytes;
-  const int acc_bufs = a.m_tiles == 1 ? 2 : 1;       // 512 columns: two buffers of 256, or one of 2 x 256
+  const int acc_bufs = m_tiles == 1 ? 2 : 1;         // 512 columns: two buffers of 256, or one of 2 x 256
   constexpr uint32_t kTmemCols = 512;
   const int n_gemm = 4 * a.n_layers + 1;
 
@@ -1297,7 +1299,7 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
           }
           if (!ok) break;
           const int stage = gi % S;
-          for (int mt = 0; mt < a.m_tiles; ++mt)
+          for (int mt = 0; mt < m_tiles; ++mt)
             tma_load_2d(x0 + (uint32_t)stage * x_bytes + (uint32_t)mt * x_tile_bytes, mp, smem_u32(&sm->full[stage]),
                         (int)(it % gs.kb) * kTileK, mt * 128, hint_x);
         }
@@ -1307,7 +1309,7 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
     // ===================== MMA issuer =====================
     if (lane == 0) {
       // M = token lanes (64 up to 64 rows: half the tensor-core work on unused lanes), N = 256 weight rows
-      const uint32_t idesc = umma_idesc_bf16(kTileN, a.NT <= 64 ? 64 : 128);
+      const uint32_t idesc = umma_idesc_bf16(kTileN, WIDE ? 128 : 64);
       int gi = 0, seg = 0;
       bool ok = true;
       for (int gm = 0; gm < n_gemm && ok; ++gm) {
@@ -1332,7 +1334,7 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
             if (!ok) break;
             tc_fence_after();
             const uint64_t dw = smem_desc_sw128(w0 + (uint32_t)stage * kBlockBytes);
-            for (int mt = 0; mt < a.m_tiles; ++mt) {
+            for (int mt = 0; mt < m_tiles; ++mt) {
               const uint64_t dx = smem_desc_sw128(x0 + (uint32_t)stage * x_bytes + (uint32_t)mt * x_tile_bytes);
 #pragma unroll
               for (int k = 0; k < kTileK / 16; ++k)
@@ -1354,7 +1356,6 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
     const int wid = wtid >> 5;
     const int quarter = warp & 3;                   // tensor-memory lane quarter this warp may read
     const int colhalf = wid >> 2;                   // warps 3-6 take the first 128 weight rows of a tile
-    const int acc_bufs = a.m_tiles == 1 ? 2 : 1;
     unsigned long long epoch = 0;
     int seg = 0;
     bool ok = true;
@@ -1389,9 +1390,9 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
         if (!ok) break;
         tc_fence_after();
         const size_t slot = (size_t)cta * gs.max_seg + seg_local;
-        for (int mt = 0; mt < a.m_tiles; ++mt) {
+        for (int mt = 0; mt < m_tiles; ++mt) {
           // batch row held by this thread's lane: 32 per lane quarter, or 16 with the 64-row instruction
-          const int per_q = a.NT <= 64 ? 16 : 32;
+          constexpr int per_q = WIDE ? 32 : 16;
           if (mt * 128 + quarter * per_q >= a.B) continue;     // no batch row in this warp's lanes (warp-uniform)
           const int tok = lane < per_q ? mt * 128 + quarter * per_q + lane : a.B;
           const uint32_t taddr =
