@@ -1168,7 +1168,8 @@ __device__ void stage_final(const MegaArgs& a, int wtid) {
 // WIDE: the variant for batches of more than 64 rows, which adds attention_warp_pairs.  It is an instantiation of
 // its own because the batches up to 64 rows live on this kernel's register allocation: the same code with the
 // extra path compiled in ran the 16-row step 2.5 % slower.
-template <int DH, bool WIDE>
+// TRACE: with the stage-boundary time stamps of CTA 0 (ss_set_trace); the timed paths run the variant without them.
+template <int DH, bool WIDE, bool TRACE>
 __global__ void __launch_bounds__(kMegaThreads, 1)
 decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_o,
                         const __grid_constant__ CUtensorMap map_act, const __grid_constant__ MegaArgs a) {
@@ -1360,7 +1361,7 @@ decode_step_mega_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_
     int seg = 0;
     bool ok = true;
 
-    const bool tracer = cta == 0 && wtid == 0 && a.trace != nullptr;
+    const bool tracer = TRACE && cta == 0 && wtid == 0 && a.trace != nullptr;
     int tr = 0;
     if (tracer) a.trace[tr++] = global_timer_ns();
     if (cta == 0 && wtid == 0) a.st.scalars[1] = 0;   // rows still active after this step (counted in the last stage)

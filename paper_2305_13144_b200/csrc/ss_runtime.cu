@@ -497,6 +497,16 @@ double weight_bytes_per_step(const ss_model_cfg& m) {
 }
 double kv_bytes_per_token(const ss_model_cfg& m) { return 2.0 * m.d_model * 2.0 * m.n_layers; }
 
+// The decode kernel's instantiations: head size 64 / 128, batches up to 64 rows / wider, without / with the stage trace.
+template <int DH>
+const void* mega_kernel_fn_dh(bool wide, bool trace) {
+  if (wide) return trace ? (const void*)decode_step_mega_kernel<DH, true, true> : (const void*)decode_step_mega_kernel<DH, true, false>;
+  return trace ? (const void*)decode_step_mega_kernel<DH, false, true> : (const void*)decode_step_mega_kernel<DH, false, false>;
+}
+const void* mega_kernel_fn(int head_dim, bool wide, bool trace) {
+  return head_dim == 128 ? mega_kernel_fn_dh<128>(wide, trace) : mega_kernel_fn_dh<64>(wide, trace);
+}
+
 // ------------------------------------------------------------------------------------ decode step
 // One cooperative launch of the persistent kernel (see ss_decode_mega.cuh).
 int enqueue_decode_step(ss_ctx* c, const ss_step_opts* opts, int32_t* next_tokens) {
@@ -551,9 +561,7 @@ int enqueue_decode_step(ss_ctx* c, const ss_step_opts* opts, int32_t* next_token
   a.wait_limit = c->wait_limit;
   void* args[4] = {(void*)mx, (void*)mo, (void*)ma, (void*)&a};
   const bool wide = NT > 64;
-  const void* fn = m.head_dim == 128
-                       ? (wide ? (const void*)decode_step_mega_kernel<128, true> : (const void*)decode_step_mega_kernel<128, false>)
-                       : (wide ? (const void*)decode_step_mega_kernel<64, true> : (const void*)decode_step_mega_kernel<64, false>);
+  const void* fn = mega_kernel_fn(m.head_dim, wide, a.trace != nullptr);
   SS_CUDA(c, cudaLaunchCooperativeKernel(fn, dim3(c->n_sm), dim3(kMegaThreads), args, smem, c->stream));
   c->grid_epochs += 1 + 2 * (unsigned long long)(4 * m.n_layers + 1);
   c->launches++;
@@ -794,14 +802,9 @@ int ss_create(const ss_model_cfg* model, const ss_runtime_cfg* rt, void* dev_are
     e = cudaFuncSetAttribute(gemm_wx_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e == cudaSuccess)
     e = cudaFuncSetAttribute(gemm_wx_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(decode_step_mega_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(decode_step_mega_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(decode_step_mega_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-  if (e == cudaSuccess)
-    e = cudaFuncSetAttribute(decode_step_mega_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  for (int v = 0; v < 8 && e == cudaSuccess; ++v)
+    e = cudaFuncSetAttribute(mega_kernel_fn((v & 1) ? 128 : 64, (v & 2) != 0, (v & 4) != 0), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             227 * 1024);
   if (e != cudaSuccess) {
     c->last_cuda = (int)e;
     delete c;
